@@ -1,0 +1,18 @@
+"""B200-native SpGEMM (gMAGNUS hot path): thin Python binding over the C ABI in include/gmagnus.h.
+
+Every step of the computation runs in the CUDA library; this package only marshals arguments.
+torch is used for device memory and streams.
+"""
+from .binding import (  # noqa: F401
+    GmError,
+    PlanOpts,
+    Plan,
+    DeviceCSR,
+    planner_params,
+    spgemm_plan,
+    spgemm_execute,
+    spgemm,
+    spgemm_host,
+    load_library,
+    EXPORTED_SYMBOLS,
+)

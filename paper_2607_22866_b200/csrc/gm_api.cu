@@ -1,0 +1,901 @@
+// C ABI of the library (see include/gmagnus.h): plan = setup phase of Algorithm 3, execute = the
+// light and heavy paths, batching of the heavy rows and assembly of C.
+#include <algorithm>
+#include <climits>
+#include <cstdio>
+#include <cstdlib>
+#include <cstring>
+#include <string>
+#include <vector>
+
+#include "gm_common.cuh"
+#include "gm_k1_analysis.cuh"
+#include "gm_k3_light.cuh"
+#include "gm_k4_expand.cuh"
+#include "gm_k5_multisplit.cuh"
+#include "gm_k6_accumulate.cuh"
+#include "gm_planner.h"
+#include "gm_scan.cuh"
+#include "gmagnus.h"
+
+namespace gm {
+
+// ------------------------------------------------------------------------------------------------
+// errors, allocator
+// ------------------------------------------------------------------------------------------------
+static thread_local std::string g_last_error;
+
+static int fail(int code, const std::string& msg) {
+  g_last_error = msg;
+  return code;
+}
+
+#define GM_CUDA(expr)                                                                              \
+  do {                                                                                             \
+    cudaError_t e_ = (expr);                                                                       \
+    if (e_ != cudaSuccess)                                                                         \
+      return fail(GM_ERR_CUDA, std::string(#expr) + ": " + cudaGetErrorString(e_));               \
+  } while (0)
+
+#define GM_TRY(expr)                \
+  do {                              \
+    int rc_ = (expr);               \
+    if (rc_ != GM_OK) return rc_;   \
+  } while (0)
+
+struct Allocator {
+  gm_alloc_fn alloc = nullptr;
+  gm_free_fn free = nullptr;
+  void* user = nullptr;
+};
+static Allocator g_alloc;
+
+static void* default_alloc(size_t bytes, cudaStream_t st) {
+  static bool pool_ready = false;
+  if (!pool_ready) {
+    int dev = 0;
+    cudaMemPool_t pool;
+    if (cudaGetDevice(&dev) == cudaSuccess && cudaDeviceGetDefaultMemPool(&pool, dev) == cudaSuccess) {
+      unsigned long long thr = ~0ull;  // keep freed blocks cached: repeated plans reuse them
+      cudaMemPoolSetAttribute(pool, cudaMemPoolAttrReleaseThreshold, &thr);
+    }
+    pool_ready = true;
+  }
+  void* p = nullptr;
+  if (cudaMallocAsync(&p, bytes, st) != cudaSuccess) {
+    cudaGetLastError();
+    return nullptr;
+  }
+  return p;
+}
+
+static void* dev_alloc(size_t bytes, cudaStream_t st) {
+  if (bytes == 0) bytes = 16;
+  if (g_alloc.alloc) return g_alloc.alloc(bytes, st, g_alloc.user);
+  return default_alloc(bytes, st);
+}
+static void dev_free(void* p, cudaStream_t st) {
+  if (!p) return;
+  if (g_alloc.free) g_alloc.free(p, st, g_alloc.user);
+  else cudaFreeAsync(p, st);
+}
+
+struct Buf {
+  void* p = nullptr;
+  size_t bytes = 0;
+  template <typename T> T* as() const { return static_cast<T*>(p); }
+};
+
+// ------------------------------------------------------------------------------------------------
+// plan
+// ------------------------------------------------------------------------------------------------
+struct PhaseTimes {
+  enum Phase { kLightSym, kLightNum, kExpand, kHist, kSplit, kAccSym, kAccNum, kScan, kCount };
+  struct Rec { int phase; cudaEvent_t a, b; };
+  std::vector<Rec> recs;
+  std::vector<cudaEvent_t> pool;
+  size_t used = 0;
+  bool enabled = false;
+  cudaEvent_t get() {
+    if (used == pool.size()) { cudaEvent_t e; cudaEventCreate(&e); pool.push_back(e); }
+    return pool[used++];
+  }
+  void begin(int phase, cudaStream_t st) {
+    if (!enabled) return;
+    Rec r{phase, get(), get()};
+    cudaEventRecord(r.a, st);
+    recs.push_back(r);
+  }
+  void end(cudaStream_t st) {
+    if (!enabled) return;
+    cudaEventRecord(recs.back().b, st);
+  }
+  void reset() { recs.clear(); used = 0; }
+  void collect(float* out) {
+    for (int i = 0; i < kCount; ++i) out[i] = 0.f;
+    for (auto& r : recs) { float ms = 0.f; cudaEventElapsedTime(&ms, r.a, r.b); out[r.phase] += ms; }
+  }
+  ~PhaseTimes() { for (auto e : pool) cudaEventDestroy(e); }
+};
+
+}  // namespace gm
+
+struct gm_plan {
+  gm_csr A{}, B{};
+  int sv = 4;
+  size_t smem_bytes = 0;
+  gm_plan_opts opts{};
+  gm_plan_info info{};
+  gm_exec_stats stats{};
+  int num_sms = 148;
+  cudaStream_t plan_stream = nullptr;
+  gm::LightBins bins{};
+  int bin_slots[gm::kMaxLightBins]{};
+  std::vector<gm::Batch> batches;
+  std::vector<int32_t> x_heavy_host;
+  int64_t max_batch_rows = 0;
+  int64_t n_seg = 0;
+  std::vector<gm::Buf> owned;
+  // device arrays
+  int64_t* nz_off = nullptr;       // nnzA + 1
+  int64_t* ip = nullptr;           // nA
+  int32_t* heavy_flag = nullptr;   // nA
+  int32_t* x_heavy = nullptr;      // nH
+  int64_t* heavy_base = nullptr;   // nH + 1
+  int64_t* seg_off = nullptr;      // n_seg + 1
+  int64_t* seg_bstart = nullptr;   // n_seg
+  int64_t* seg_j = nullptr;        // n_seg
+  int64_t* heavy_nz_off = nullptr; // nH + 1
+  int32_t* sym_rows = nullptr;     // bins x nA
+  int* sym_fill = nullptr;         // 8
+  int32_t* num_rows = nullptr;     // bins x nA
+  int* num_fill = nullptr;         // 8
+  int32_t* row_nnz = nullptr;      // nA
+  int64_t* scan_tmp = nullptr;
+  int64_t* c_total = nullptr;      // running nnz(C) (device carry)
+  int* err = nullptr;
+  // heavy workspace
+  int32_t* stage_col[2]{};
+  void* stage_val[2]{};
+  gm::u32* counts = nullptr;       // max_batch_rows * chunks_required
+  gm::u64* cursor = nullptr;       // same
+  int64_t* level_off[2]{};         // max_batch_rows * chunks_required + 1 each (ping-pong)
+  gm::u32* chunk_nnz = nullptr;
+  int64_t* chunk_nnz_off = nullptr;
+  gm::PhaseTimes times;
+};
+
+namespace gm {
+
+template <typename T>
+static int plan_alloc(gm_plan* p, T** out, size_t n, cudaStream_t st) {
+  Buf b;
+  b.bytes = n * sizeof(T);
+  b.p = dev_alloc(b.bytes, st);
+  if (!b.p) return fail(GM_ERR_OOM, "device allocation of " + std::to_string(b.bytes) + " bytes failed");
+  p->owned.push_back(b);
+  p->info.workspace_bytes += static_cast<int64_t>(b.bytes);
+  *out = static_cast<T*>(b.p);
+  return GM_OK;
+}
+
+static unsigned grid_for(i64 n, int threads, int num_sms, int per_sm = 16) {
+  i64 g = (n + threads - 1) / threads;
+  const i64 cap = static_cast<i64>(num_sms) * per_sm;
+  if (g > cap) g = cap;
+  if (g < 1) g = 1;
+  return static_cast<unsigned>(g);
+}
+
+static int check_csr_arg(const gm_csr* M, const char* name) {
+  if (!M) return fail(GM_ERR_INVALID_ARG, std::string(name) + " is null");
+  if (M->n_rows < 0 || M->n_cols < 0 || M->nnz < 0 || M->n_cols > INT32_MAX || M->n_rows > INT32_MAX)
+    return fail(GM_ERR_INVALID_ARG, std::string(name) + ": sizes out of range");
+  if (!M->row_ptr || (M->nnz > 0 && (!M->col_idx || !M->vals)))
+    return fail(GM_ERR_INVALID_ARG, std::string(name) + ": null array");
+  if (M->dtype != GM_F32 && M->dtype != GM_F64) return fail(GM_ERR_DTYPE, std::string(name) + ": unknown dtype");
+  return GM_OK;
+}
+
+__global__ void k_validate_csr(const i64* __restrict__ row_ptr, const int32_t* __restrict__ col, i64 n_rows, i64 n_cols,
+                               i64 nnz, int* __restrict__ bad) {
+  for (i64 i = static_cast<i64>(blockIdx.x) * blockDim.x + threadIdx.x; i < n_rows;
+       i += static_cast<i64>(gridDim.x) * blockDim.x) {
+    const i64 s = row_ptr[i], e = row_ptr[i + 1];
+    if ((i == 0 && s != 0) || e < s || e > nnz || (i == n_rows - 1 && e != nnz)) { *bad = 1; continue; }
+    for (i64 k = s; k < e; ++k) {
+      const int32_t c = col[k];
+      if (c < 0 || c >= n_cols || (k > s && col[k - 1] >= c)) { *bad = 1; break; }
+    }
+  }
+}
+
+static int build_plan(gm_plan* p, cudaStream_t st) {
+  const gm_csr& A = p->A;
+  const gm_csr& B = p->B;
+  const i64 nA = A.n_rows, nnzA = A.nnz;
+  gm_plan_info& info = p->info;
+  info.n_rows = nA;
+  info.n_cols_c = B.n_cols;
+
+  int dev = 0;
+  GM_CUDA(cudaGetDevice(&dev));
+  cudaDeviceProp prop;
+  GM_CUDA(cudaGetDeviceProperties(&prop, dev));
+  p->num_sms = prop.multiProcessorCount;
+  if (p->smem_bytes > prop.sharedMemPerBlockOptin)
+    return fail(GM_ERR_UNSUPPORTED_SMEM, "smem_bytes exceeds the device's opt-in shared memory per block");
+  {
+    const int rc = planner_params(B.n_cols, A.dtype, p->smem_bytes, &p->opts, &info.params);
+    if (rc != GM_OK) return fail(rc, "planner rejected the parameters");
+  }
+  const gm_params& prm = info.params;
+
+  GM_TRY(plan_alloc(p, &p->err, 4, st));
+  GM_CUDA(cudaMemsetAsync(p->err, 0, 4 * sizeof(int), st));
+  if (p->opts.validate_inputs) {
+    for (const gm_csr* M : {&A, &B}) {
+      if (M->n_rows == 0) continue;
+      k_validate_csr<<<grid_for(M->n_rows, 256, p->num_sms), 256, 0, st>>>(M->row_ptr, M->col_idx, M->n_rows,
+                                                                          M->n_cols, M->nnz, p->err + 1);
+    }
+    int bad = 0;
+    GM_CUDA(cudaMemcpyAsync(&bad, p->err + 1, sizeof(int), cudaMemcpyDeviceToHost, st));
+    GM_CUDA(cudaStreamSynchronize(st));
+    if (bad) return fail(GM_ERR_BAD_CSR, "row_ptr not monotone / columns out of range or not strictly ascending");
+  }
+
+  // ---- K1: products per stored entry, flattened product space, products per row
+  int32_t* nz_len = nullptr;
+  K1Totals* totals = nullptr;
+  int64_t* heavy_pos = nullptr;
+  GM_TRY(plan_alloc(p, &nz_len, static_cast<size_t>(nnzA) + 1, st));
+  GM_TRY(plan_alloc(p, &p->nz_off, static_cast<size_t>(nnzA) + 1, st));
+  GM_TRY(plan_alloc(p, &p->ip, static_cast<size_t>(nA) + 1, st));
+  GM_TRY(plan_alloc(p, &p->heavy_flag, static_cast<size_t>(nA) + 1, st));
+  GM_TRY(plan_alloc(p, &heavy_pos, static_cast<size_t>(nA) + 1, st));
+  GM_TRY(plan_alloc(p, &totals, 1, st));
+  GM_TRY(plan_alloc(p, &p->row_nnz, static_cast<size_t>(nA) + 1, st));
+  GM_TRY(plan_alloc(p, &p->c_total, 2, st));
+  GM_TRY(plan_alloc(p, &p->scan_tmp, static_cast<size_t>(scan_tmp_elems(std::max<i64>(std::max(nnzA, nA), 1))), st));
+  GM_CUDA(cudaMemsetAsync(totals, 0, sizeof(K1Totals), st));
+  if (nnzA > 0) k1_nz_len<<<grid_for(nnzA, 256, p->num_sms, 32), 256, 0, st>>>(A.col_idx, nnzA, B.row_ptr, nz_len);
+  exclusive_scan<int32_t, i64>(nz_len, p->nz_off, nnzA, p->scan_tmp, nullptr, nullptr, nullptr, st);
+  if (nA > 0) {
+    k1_row_products<<<grid_for(nA, 256, p->num_sms), 256, 0, st>>>(A.row_ptr, nA, p->nz_off, prm.tau, B.n_cols, p->ip,
+                                                                  p->heavy_flag, totals);
+  }
+  exclusive_scan<int32_t, i64>(p->heavy_flag, heavy_pos, nA, p->scan_tmp, nullptr, nullptr, nullptr, st);
+
+  // ---- light rows: bins by IP_i for the symbolic pass
+  {
+    const int top_cap = static_cast<int>(pow2_ceil(static_cast<uint64_t>(std::max<i64>(prm.tau, 16))));
+    const int std_caps[] = {16, 64, 256, 1024, 4096, 16384, 65536};
+    int nb = 0;
+    for (int c : std_caps)
+      if (c < top_cap && nb < kMaxLightBins - 1) { p->bins.cap[nb] = c; p->bin_slots[nb] = 2 * c; ++nb; }
+    p->bins.cap[nb] = top_cap;
+    p->bin_slots[nb] = prm.light_slots;
+    p->bins.n_bins = nb + 1;
+  }
+  GM_TRY(plan_alloc(p, &p->sym_rows, static_cast<size_t>(p->bins.n_bins) * static_cast<size_t>(std::max<i64>(nA, 1)), st));
+  GM_TRY(plan_alloc(p, &p->num_rows, static_cast<size_t>(p->bins.n_bins) * static_cast<size_t>(std::max<i64>(nA, 1)), st));
+  GM_TRY(plan_alloc(p, &p->sym_fill, 8, st));
+  GM_TRY(plan_alloc(p, &p->num_fill, 8, st));
+  GM_CUDA(cudaMemsetAsync(p->sym_fill, 0, 8 * sizeof(int), st));
+  if (nA > 0) {
+    // tau may be below the top bin's capacity (forced tau): rows with tau < IP <= cap are heavy and skipped
+    k1_bin_rows<i64><<<static_cast<unsigned>((nA + 255) / 256), 256, 0, st>>>(p->ip, p->heavy_flag, nA, p->bins, nA,
+                                                                             p->sym_fill, p->sym_rows);
+  }
+
+  // ---- first host sync: totals
+  K1Totals ht{};
+  int fill[8] = {0};
+  GM_CUDA(cudaMemcpyAsync(&ht, totals, sizeof(ht), cudaMemcpyDeviceToHost, st));
+  GM_CUDA(cudaMemcpyAsync(fill, p->sym_fill, sizeof(fill), cudaMemcpyDeviceToHost, st));
+  GM_CUDA(cudaStreamSynchronize(st));
+  info.products_total = static_cast<int64_t>(ht.products_total);
+  info.products_heavy = static_cast<int64_t>(ht.products_heavy);
+  info.products_max_row = static_cast<int64_t>(ht.products_max_row);
+  info.c_nnz_upper = static_cast<int64_t>(ht.c_nnz_upper);
+  info.rows_heavy = static_cast<int64_t>(ht.rows_heavy);
+  info.rows_empty = static_cast<int64_t>(ht.rows_empty);
+  info.rows_light = nA - info.rows_heavy - info.rows_empty;
+  info.nnz_a_heavy = static_cast<int64_t>(ht.nnz_a_heavy);
+  for (int b = 0; b < 8; ++b) info.light_bin_rows[b] = fill[b];
+  const i64 nH = info.rows_heavy;
+  p->n_seg = info.nnz_a_heavy;
+
+  // ---- heavy rows: lists, prefix sums, segment table
+  if (nH > 0) {
+    int64_t *heavy_ip = nullptr, *heavy_nnz = nullptr;
+    GM_TRY(plan_alloc(p, &p->x_heavy, static_cast<size_t>(nH), st));
+    GM_TRY(plan_alloc(p, &heavy_ip, static_cast<size_t>(nH) + 1, st));
+    GM_TRY(plan_alloc(p, &heavy_nnz, static_cast<size_t>(nH) + 1, st));
+    GM_TRY(plan_alloc(p, &p->heavy_base, static_cast<size_t>(nH) + 1, st));
+    GM_TRY(plan_alloc(p, &p->heavy_nz_off, static_cast<size_t>(nH) + 1, st));
+    GM_TRY(plan_alloc(p, &p->seg_off, static_cast<size_t>(p->n_seg) + 1, st));
+    GM_TRY(plan_alloc(p, &p->seg_bstart, static_cast<size_t>(p->n_seg) + 1, st));
+    GM_TRY(plan_alloc(p, &p->seg_j, static_cast<size_t>(p->n_seg) + 1, st));
+    k1_heavy_scatter<<<grid_for(nA, 256, p->num_sms), 256, 0, st>>>(p->heavy_flag, heavy_pos, p->ip, A.row_ptr, nA,
+                                                                   p->x_heavy, heavy_ip, heavy_nnz);
+    exclusive_scan<i64, i64>(heavy_ip, p->heavy_base, nH, p->scan_tmp, nullptr, nullptr, nullptr, st);
+    exclusive_scan<i64, i64>(heavy_nnz, p->heavy_nz_off, nH, p->scan_tmp, nullptr, nullptr, nullptr, st);
+    k1_heavy_segments<<<grid_for(p->n_seg + 1, 256, p->num_sms, 32), 256, 0, st>>>(
+        p->x_heavy, nH, p->heavy_nz_off, p->heavy_base, A.row_ptr, A.col_idx, p->nz_off, B.row_ptr, p->n_seg, p->seg_off,
+        p->seg_bstart, p->seg_j);
+    std::vector<int64_t> hb(static_cast<size_t>(nH) + 1);
+    p->x_heavy_host.resize(static_cast<size_t>(nH));
+    GM_CUDA(cudaMemcpyAsync(hb.data(), p->heavy_base, hb.size() * sizeof(int64_t), cudaMemcpyDeviceToHost, st));
+    GM_CUDA(cudaMemcpyAsync(p->x_heavy_host.data(), p->x_heavy, static_cast<size_t>(nH) * sizeof(int32_t),
+                            cudaMemcpyDeviceToHost, st));
+    GM_CUDA(cudaStreamSynchronize(st));
+
+    // ---- batches: consecutive heavy rows whose products fit one staging half-buffer
+    i64 stage = p->opts.stage_elems > 0 ? p->opts.stage_elems : (i64{1} << 29);
+    if (p->opts.stage_elems == 0) stage = std::max(stage, info.products_max_row);  // a row is never split
+    stage = std::min(stage, info.products_heavy);
+    const i64 kMaxStage = (i64{1} << 31) - kSplitTile;  // batch-relative positions are 32-bit in the multisplit tiles
+    if (stage > kMaxStage) stage = kMaxStage;
+    if (info.products_max_row > stage)
+      return fail(GM_ERR_CAPACITY, "a heavy row has " + std::to_string(info.products_max_row) +
+                                       " products, more than one staging half-buffer holds (" + std::to_string(stage) + ")");
+    if (!cut_batches(hb.data(), nH, stage, &p->batches)) return fail(GM_ERR_CAPACITY, "batch cutting failed");
+    info.n_batches = static_cast<int64_t>(p->batches.size());
+    info.stage_elems = 0;
+    for (const Batch& b : p->batches) {
+      info.stage_elems = std::max(info.stage_elems, b.elems);
+      p->max_batch_rows = std::max(p->max_batch_rows, b.h1 - b.h0);
+    }
+    const size_t se = static_cast<size_t>(info.stage_elems);
+    const int n_buf = prm.n_levels > 0 ? 2 : 1;
+    for (int i = 0; i < n_buf; ++i) {
+      GM_TRY(plan_alloc(p, &p->stage_col[i], se, st));
+      unsigned char* v = nullptr;
+      GM_TRY(plan_alloc(p, &v, se * static_cast<size_t>(p->sv), st));
+      p->stage_val[i] = v;
+    }
+    const size_t n_chunks_max = static_cast<size_t>(p->max_batch_rows) * static_cast<size_t>(prm.chunks_required);
+    GM_TRY(plan_alloc(p, &p->level_off[0], n_chunks_max + 1, st));
+    if (prm.n_levels > 0) {
+      GM_TRY(plan_alloc(p, &p->counts, n_chunks_max + 1, st));
+      GM_TRY(plan_alloc(p, &p->cursor, n_chunks_max + 1, st));
+      GM_TRY(plan_alloc(p, &p->level_off[1], n_chunks_max + 1, st));
+    }
+    GM_TRY(plan_alloc(p, &p->chunk_nnz, n_chunks_max + 1, st));
+    GM_TRY(plan_alloc(p, &p->chunk_nnz_off, n_chunks_max + 1, st));
+    int64_t* tmp2 = nullptr;  // the per-batch scans can be longer than the ones above
+    GM_TRY(plan_alloc(p, &tmp2, static_cast<size_t>(scan_tmp_elems(std::max<i64>({static_cast<i64>(n_chunks_max), nnzA, nA, 1}))), st));
+    p->scan_tmp = tmp2;
+  }
+  GM_CUDA(cudaStreamSynchronize(st));
+  return GM_OK;
+}
+
+// ------------------------------------------------------------------------------------------------
+// execute
+// ------------------------------------------------------------------------------------------------
+template <typename V, bool NUMERIC, int G, int LPN, int BT>
+static int launch_light_one(gm_plan* p, const int32_t* rows, const int* n_rows_dev, i64 n_rows_upper, int slots, int cap,
+                            const i64* c_row_ptr, int32_t* c_col, V* c_val, i64 c_capacity, cudaStream_t st) {
+  constexpr int kGroups = BT / G;
+  const size_t smem = kGroups * light_group_bytes<V, NUMERIC>(slots, cap);
+  auto kern = k3_light_rows<V, G, LPN, BT, NUMERIC>;
+  if (smem > 48 * 1024) GM_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)));
+  const unsigned grid = grid_for(n_rows_upper, kGroups, p->num_sms, 2048 / BT * 4);
+  kern<<<grid, BT, smem, st>>>(p->A.row_ptr, p->A.col_idx, static_cast<const V*>(p->A.vals), p->B.row_ptr, p->B.col_idx,
+                               static_cast<const V*>(p->B.vals), rows, n_rows_dev, slots, cap, p->row_nnz, c_row_ptr, c_col,
+                               c_val, c_capacity, p->err);
+  ++p->stats.launches;
+  GM_CUDA(cudaGetLastError());
+  return GM_OK;
+}
+
+template <typename V, bool NUMERIC>
+static int launch_light(gm_plan* p, const int32_t* rows_all, const int* fill_dev, const i64* rows_upper,
+                        const i64* c_row_ptr, int32_t* c_col, V* c_val, i64 c_capacity, cudaStream_t st) {
+  const i64 stride = std::max<i64>(p->A.n_rows, 1);
+  for (int b = 0; b < p->bins.n_bins; ++b) {
+    if (rows_upper[b] <= 0) continue;
+    const int cap = p->bins.cap[b], slots = p->bin_slots[b];
+    const int32_t* rows = rows_all + static_cast<size_t>(b) * stride;
+    const int* nd = fill_dev + b;
+    const i64 up = rows_upper[b];
+#define GM_LIGHT(G, LPN, BT) launch_light_one<V, NUMERIC, G, LPN, BT>(p, rows, nd, up, slots, cap, c_row_ptr, c_col, c_val, c_capacity, st)
+    int rc;
+    if (cap <= 16) rc = GM_LIGHT(8, 1, 256);
+    else if (cap <= 64) rc = GM_LIGHT(32, 4, 256);
+    else if (cap <= 256) rc = GM_LIGHT(128, 8, 128);
+    else if (cap <= 1024) rc = GM_LIGHT(256, 16, 256);
+    else if (cap <= 4096) rc = GM_LIGHT(512, 32, 512);
+    else rc = GM_LIGHT(1024, 32, 1024);
+#undef GM_LIGHT
+    GM_TRY(rc);
+  }
+  return GM_OK;
+}
+
+__global__ void k_heavy_row_counts(const i64* __restrict__ chunk_nnz_off, int log2_chunks_per_row, i64 n_rows_b,
+                                   const int32_t* __restrict__ x_heavy, i64 h0, int32_t* __restrict__ row_nnz) {
+  for (i64 r = static_cast<i64>(blockIdx.x) * blockDim.x + threadIdx.x; r < n_rows_b;
+       r += static_cast<i64>(gridDim.x) * blockDim.x) {
+    row_nnz[x_heavy[h0 + r]] =
+        static_cast<int32_t>(chunk_nnz_off[(r + 1) << log2_chunks_per_row] - chunk_nnz_off[r << log2_chunks_per_row]);
+  }
+}
+
+__global__ void k_rebase(const i64* __restrict__ in, i64 n, i64 bias, i64* __restrict__ out) {
+  for (i64 i = static_cast<i64>(blockIdx.x) * blockDim.x + threadIdx.x; i < n;
+       i += static_cast<i64>(gridDim.x) * blockDim.x)
+    out[i] = in[i] - bias;
+}
+
+template <typename V>
+struct HeavyBatchState {
+  const int32_t* fin_col = nullptr;  // staging buffer that holds the final chunks
+  const V* fin_val = nullptr;
+  const i64* chunk_off = nullptr;    // n_chunks + 1 batch-relative offsets
+  i64 n_chunks = 0;
+  int log2_cpr = 0;
+};
+
+template <typename V, bool NUMERIC>
+static int launch_accumulate(gm_plan* p, const Batch& b, const HeavyBatchState<V>& hs, const i64* c_row_ptr,
+                             int32_t* c_col, V* c_val, i64 c_capacity, cudaStream_t st) {
+  const gm_params& prm = p->info.params;
+  const int W = prm.chunk_width;
+  const size_t smem = acc_smem_bytes(W, sizeof(V), NUMERIC);
+  const int ctas = NUMERIC ? prm.acc_ctas_per_sm : 8;
+  const unsigned grid = static_cast<unsigned>(std::min<i64>(hs.n_chunks, static_cast<i64>(p->num_sms) * ctas));
+#define GM_ACC(BT)                                                                                                    \
+  do {                                                                                                                \
+    auto kern = k6_accumulate<V, NUMERIC, BT>;                                                                        \
+    if (smem > 48 * 1024)                                                                                             \
+      GM_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)));      \
+    kern<<<grid, BT, smem, st>>>(hs.fin_col, hs.fin_val, hs.chunk_off, hs.n_chunks, hs.log2_cpr, W, p->B.n_cols,      \
+                                 p->chunk_nnz, p->chunk_nnz_off, p->x_heavy, b.h0, c_row_ptr, c_col, c_val, c_capacity, \
+                                 p->err);                                                                             \
+  } while (0)
+  if (!NUMERIC) GM_ACC(256);
+  else if (prm.acc_ctas_per_sm == 1) GM_ACC(1024);
+  else if (prm.acc_ctas_per_sm == 2) GM_ACC(512);
+  else GM_ACC(256);
+#undef GM_ACC
+  ++p->stats.launches;
+  GM_CUDA(cudaGetLastError());
+  return GM_OK;
+}
+
+// Expansion, every multisplit level and the symbolic accumulate of one batch.  Leaves C^_reord in
+// the staging buffer and the per-chunk entry counts (and their scan) in chunk_nnz / chunk_nnz_off,
+// and writes the heavy rows' entry counts into row_nnz.
+template <typename V>
+static int heavy_batch_front(gm_plan* p, const Batch& b, HeavyBatchState<V>* hs, cudaStream_t st) {
+  const gm_params& prm = p->info.params;
+  const i64 rows_b = b.h1 - b.h0;
+  PhaseTimes& tm = p->times;
+  tm.begin(PhaseTimes::kExpand, st);
+  {
+    const unsigned grid = static_cast<unsigned>((b.elems + kExpandTile - 1) / kExpandTile);
+    k4_expand<V><<<grid, kExpandThreads, 0, st>>>(p->seg_off, p->seg_bstart, p->seg_j, 0, p->n_seg,
+                                                  static_cast<const V*>(p->A.vals), p->B.col_idx,
+                                                  static_cast<const V*>(p->B.vals), b.elem0, b.elems, p->stage_col[0],
+                                                  static_cast<V*>(p->stage_val[0]));
+    ++p->stats.launches;
+    GM_CUDA(cudaGetLastError());
+  }
+  tm.end(st);
+  // level-0 parents are the batch's rows: offsets relative to the batch
+  i64* off_cur = p->level_off[0];
+  i64* off_nxt = p->level_off[1];
+  k_rebase<<<grid_for(rows_b + 1, 256, p->num_sms), 256, 0, st>>>(p->heavy_base + b.h0, rows_b + 1, b.elem0, off_cur);
+  ++p->stats.launches;
+  int cur = 0;
+  i64 n_par = rows_b;
+  if (prm.n_levels > 0) {
+    GM_CUDA(cudaFuncSetAttribute(k5_level<V, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 static_cast<int>(split_smem_bytes<V>(true))));
+  }
+  for (int l = 0; l < prm.n_levels; ++l) {
+    const int F = prm.fanout[l];
+    const i64 n_child = n_par * F;
+    const unsigned grid = static_cast<unsigned>((b.elems + kSplitTile - 1) / kSplitTile);
+    const int32_t* xc = p->stage_col[cur];
+    const V* xv = static_cast<const V*>(p->stage_val[cur]);
+    tm.begin(PhaseTimes::kHist, st);
+    GM_CUDA(cudaMemsetAsync(p->counts, 0, static_cast<size_t>(n_child) * sizeof(u32), st));
+    k5_level<V, false><<<grid, kSplitThreads, split_smem_bytes<V>(false), st>>>(
+        xc, xv, b.elems, off_cur, n_par, F, prm.shift[l], p->counts, nullptr, nullptr, nullptr);
+    ++p->stats.launches;
+    GM_CUDA(cudaGetLastError());
+    tm.end(st);
+    tm.begin(PhaseTimes::kScan, st);
+    exclusive_scan<u32, i64>(p->counts, off_nxt, n_child, p->scan_tmp, nullptr, nullptr, reinterpret_cast<i64*>(p->cursor), st);
+    p->stats.launches += 3;
+    tm.end(st);
+    tm.begin(PhaseTimes::kSplit, st);
+    k5_level<V, true><<<grid, kSplitThreads, split_smem_bytes<V>(true), st>>>(
+        xc, xv, b.elems, off_cur, n_par, F, prm.shift[l], nullptr, p->cursor, p->stage_col[cur ^ 1],
+        static_cast<V*>(p->stage_val[cur ^ 1]));
+    ++p->stats.launches;
+    GM_CUDA(cudaGetLastError());
+    tm.end(st);
+    std::swap(off_cur, off_nxt);
+    cur ^= 1;
+    n_par = n_child;
+  }
+  hs->fin_col = p->stage_col[cur];
+  hs->fin_val = static_cast<const V*>(p->stage_val[cur]);
+  hs->chunk_off = off_cur;
+  hs->n_chunks = n_par;
+  hs->log2_cpr = ilog2_floor(static_cast<uint64_t>(prm.chunks_required));
+  p->stats.final_chunks += n_par;
+  p->stats.staged_products += b.elems;
+
+  tm.begin(PhaseTimes::kAccSym, st);
+  GM_TRY((launch_accumulate<V, false>(p, b, *hs, nullptr, nullptr, nullptr, 0, st)));
+  tm.end(st);
+  tm.begin(PhaseTimes::kScan, st);
+  exclusive_scan<u32, i64>(p->chunk_nnz, p->chunk_nnz_off, hs->n_chunks, p->scan_tmp, nullptr, nullptr, nullptr, st);
+  k_heavy_row_counts<<<grid_for(rows_b, 256, p->num_sms), 256, 0, st>>>(p->chunk_nnz_off, hs->log2_cpr, rows_b, p->x_heavy,
+                                                                        b.h0, p->row_nnz);
+  p->stats.launches += 4;
+  tm.end(st);
+  return GM_OK;
+}
+
+static int dev_error_to_status(int code) {
+  switch (code) {
+    case kDevOk: return GM_OK;
+    case kDevCapacity: return fail(GM_ERR_CAPACITY, "C did not fit the room reserved for it (raise c_capacity or stage fewer products)");
+    case kDevTableFull: return fail(GM_ERR_INTERNAL, "a light-row hash table overflowed");
+    case kDevBadChunk: return fail(GM_ERR_INTERNAL, "an intermediate product reached a chunk that does not own its column");
+    default: return fail(GM_ERR_INTERNAL, "unknown device error code");
+  }
+}
+
+template <typename V>
+static int execute_t(gm_plan* p, cudaStream_t st, gm_csr* C) {
+  const gm_csr& A = p->A;
+  const gm_csr& B = p->B;
+  const i64 nA = A.n_rows;
+  gm_plan_info& info = p->info;
+  PhaseTimes& tm = p->times;
+  p->stats = gm_exec_stats{};
+  tm.reset();
+  cudaEvent_t ev_total0 = nullptr, ev_total1 = nullptr;
+  if (tm.enabled) { ev_total0 = tm.get(); ev_total1 = tm.get(); cudaEventRecord(ev_total0, st); }
+
+  GM_CUDA(cudaMemsetAsync(p->err, 0, sizeof(int), st));
+  GM_CUDA(cudaMemsetAsync(p->row_nnz, 0, static_cast<size_t>(nA + 1) * sizeof(int32_t), st));
+  GM_CUDA(cudaMemsetAsync(p->c_total, 0, 2 * sizeof(int64_t), st));
+
+  // ---- result row_ptr
+  i64* c_row_ptr = static_cast<i64*>(dev_alloc(static_cast<size_t>(nA + 1) * sizeof(i64), st));
+  if (!c_row_ptr) return fail(GM_ERR_OOM, "allocation of C.row_ptr failed");
+  int32_t* c_col = nullptr;
+  V* c_val = nullptr;
+  auto cleanup = [&]() {
+    dev_free(c_row_ptr, st);
+    dev_free(c_col, st);
+    dev_free(c_val, st);
+  };
+#define GM_TRY_C(expr) do { int rc2_ = (expr); if (rc2_ != GM_OK) { cudaStreamSynchronize(st); cleanup(); return rc2_; } } while (0)
+
+  // ---- light rows, symbolic (Algorithm 3: Symbolic(A[x_light,:], B))
+  tm.begin(PhaseTimes::kLightSym, st);
+  GM_TRY_C((launch_light<V, false>(p, p->sym_rows, p->sym_fill, info.light_bin_rows, nullptr, nullptr, nullptr, 0, st)));
+  tm.end(st);
+
+  // a row's numeric bin is never above its symbolic bin
+  i64 num_upper[kMaxLightBins] = {0};
+  {
+    i64 run = 0;
+    for (int b = p->bins.n_bins - 1; b >= 0; --b) { run += info.light_bin_rows[b]; num_upper[b] = run; }
+  }
+  auto light_numeric = [&](i64 capacity) -> int {
+    tm.begin(PhaseTimes::kLightNum, st);
+    if (info.rows_light > 0) {
+      GM_CUDA(cudaMemsetAsync(p->num_fill, 0, 8 * sizeof(int), st));
+      k1_bin_rows<int32_t><<<static_cast<unsigned>((nA + 255) / 256), 256, 0, st>>>(p->row_nnz, p->heavy_flag, nA, p->bins,
+                                                                                    std::max<i64>(nA, 1), p->num_fill, p->num_rows);
+      ++p->stats.launches;
+      GM_TRY((launch_light<V, true>(p, p->num_rows, p->num_fill, num_upper, c_row_ptr, c_col, c_val, capacity, st)));
+    }
+    tm.end(st);
+    return GM_OK;
+  };
+
+  const size_t n_batches = p->batches.size();
+  i64 capacity = 0;
+  i64 total = 0;
+  int dev_err = 0;
+  if (n_batches <= 1) {
+    // ---- everything is resident at once: count, allocate C exactly, then fill
+    HeavyBatchState<V> hs;
+    if (n_batches == 1) GM_TRY_C(heavy_batch_front<V>(p, p->batches[0], &hs, st));
+    tm.begin(PhaseTimes::kScan, st);
+    exclusive_scan<int32_t, i64>(p->row_nnz, c_row_ptr, nA, p->scan_tmp, nullptr, p->c_total, nullptr, st);
+    p->stats.launches += 3;
+    tm.end(st);
+    if (cudaMemcpyAsync(&total, p->c_total, sizeof(i64), cudaMemcpyDeviceToHost, st) != cudaSuccess ||
+        cudaStreamSynchronize(st) != cudaSuccess) {
+      cleanup();
+      return fail(GM_ERR_CUDA, std::string("symbolic phase failed: ") + cudaGetErrorString(cudaGetLastError()));
+    }
+    capacity = total;
+    c_col = static_cast<int32_t*>(dev_alloc(static_cast<size_t>(std::max<i64>(total, 1)) * sizeof(int32_t), st));
+    c_val = static_cast<V*>(dev_alloc(static_cast<size_t>(std::max<i64>(total, 1)) * sizeof(V), st));
+    if (!c_col || !c_val) { cleanup(); return fail(GM_ERR_OOM, "allocation of C (" + std::to_string(total) + " entries) failed"); }
+    if (n_batches == 1) {
+      tm.begin(PhaseTimes::kAccNum, st);
+      GM_TRY_C((launch_accumulate<V, true>(p, p->batches[0], hs, c_row_ptr, c_col, c_val, capacity, st)));
+      tm.end(st);
+    }
+    GM_TRY_C(light_numeric(capacity));
+  } else {
+    // ---- heavy rows in several staging-buffer fills: C is appended in row order into reserved room
+    capacity = p->opts.c_capacity;
+    if (capacity <= 0) {
+      size_t free_b = 0, total_b = 0;
+      GM_CUDA(cudaMemGetInfo(&free_b, &total_b));
+      const i64 reserve = i64{1} << 30;
+      const i64 by_mem = (static_cast<i64>(free_b) - reserve - (nA + 1) * 8) / static_cast<i64>(4 + sizeof(V));
+      capacity = std::min<i64>(info.c_nnz_upper, std::max<i64>(by_mem, 1));
+    }
+    c_col = static_cast<int32_t*>(dev_alloc(static_cast<size_t>(std::max<i64>(capacity, 1)) * sizeof(int32_t), st));
+    c_val = static_cast<V*>(dev_alloc(static_cast<size_t>(std::max<i64>(capacity, 1)) * sizeof(V), st));
+    if (!c_col || !c_val) { cleanup(); return fail(GM_ERR_OOM, "allocation of C (room for " + std::to_string(capacity) + " entries) failed"); }
+    for (size_t bi = 0; bi < n_batches; ++bi) {
+      const Batch& b = p->batches[bi];
+      HeavyBatchState<V> hs;
+      GM_TRY_C(heavy_batch_front<V>(p, b, &hs, st));
+      // rows [r0, r1) of C get their offsets now: every light row in the range was counted up front
+      const i64 r0 = bi == 0 ? 0 : p->x_heavy_host[static_cast<size_t>(b.h0)];
+      const i64 r1 = bi + 1 == n_batches ? nA : p->x_heavy_host[static_cast<size_t>(p->batches[bi + 1].h0)];
+      tm.begin(PhaseTimes::kScan, st);
+      exclusive_scan<int32_t, i64>(p->row_nnz + r0, c_row_ptr + r0, r1 - r0, p->scan_tmp, p->c_total, p->c_total, nullptr, st);
+      p->stats.launches += 3;
+      tm.end(st);
+      tm.begin(PhaseTimes::kAccNum, st);
+      GM_TRY_C((launch_accumulate<V, true>(p, b, hs, c_row_ptr, c_col, c_val, capacity, st)));
+      tm.end(st);
+    }
+    GM_TRY_C(light_numeric(capacity));
+    if (cudaMemcpyAsync(&total, p->c_total, sizeof(i64), cudaMemcpyDeviceToHost, st) != cudaSuccess) {
+      cleanup();
+      return fail(GM_ERR_CUDA, "copy of nnz(C) failed");
+    }
+  }
+  if (tm.enabled) cudaEventRecord(ev_total1, st);
+  cudaError_t e1 = cudaMemcpyAsync(&dev_err, p->err, sizeof(int), cudaMemcpyDeviceToHost, st);
+  cudaError_t e2 = cudaStreamSynchronize(st);
+  if (e1 != cudaSuccess || e2 != cudaSuccess) {
+    cleanup();
+    return fail(GM_ERR_CUDA, std::string("execute failed: ") + cudaGetErrorString(e2 != cudaSuccess ? e2 : e1));
+  }
+  if (dev_err != kDevOk || total > capacity) {
+    cleanup();
+    if (dev_err == kDevOk) dev_err = kDevCapacity;
+    return dev_error_to_status(dev_err);
+  }
+#undef GM_TRY_C
+  p->stats.c_nnz = total;
+  p->stats.c_capacity = capacity;
+  if (tm.enabled) {
+    float ph[PhaseTimes::kCount];
+    tm.collect(ph);
+    p->stats.ms_light_symbolic = ph[PhaseTimes::kLightSym];
+    p->stats.ms_light_numeric = ph[PhaseTimes::kLightNum];
+    p->stats.ms_expand = ph[PhaseTimes::kExpand];
+    p->stats.ms_histogram = ph[PhaseTimes::kHist];
+    p->stats.ms_multisplit = ph[PhaseTimes::kSplit];
+    p->stats.ms_acc_symbolic = ph[PhaseTimes::kAccSym];
+    p->stats.ms_acc_numeric = ph[PhaseTimes::kAccNum];
+    p->stats.ms_scan = ph[PhaseTimes::kScan];
+    cudaEventElapsedTime(&p->stats.ms_total, ev_total0, ev_total1);
+  }
+  C->n_rows = nA;
+  C->n_cols = B.n_cols;
+  C->nnz = total;
+  C->row_ptr = c_row_ptr;
+  C->col_idx = c_col;
+  C->vals = c_val;
+  C->dtype = A.dtype;
+  C->reserved = 0;
+  return GM_OK;
+}
+
+}  // namespace gm
+
+// ------------------------------------------------------------------------------------------------
+// extern "C"
+// ------------------------------------------------------------------------------------------------
+using namespace gm;
+
+extern "C" {
+
+int gm_set_allocator(gm_alloc_fn alloc_fn, gm_free_fn free_fn, void* user) {
+  if ((alloc_fn == nullptr) != (free_fn == nullptr)) return fail(GM_ERR_INVALID_ARG, "alloc and free must be given together");
+  g_alloc.alloc = alloc_fn;
+  g_alloc.free = free_fn;
+  g_alloc.user = user;
+  return GM_OK;
+}
+
+int gm_spgemm_plan_ex(const gm_csr* A, const gm_csr* B, size_t smem_bytes, const gm_plan_opts* opts, void* cuda_stream,
+                      gm_plan** plan_out) {
+  if (!plan_out) return fail(GM_ERR_INVALID_ARG, "plan_out is null");
+  *plan_out = nullptr;
+  GM_TRY(check_csr_arg(A, "A"));
+  GM_TRY(check_csr_arg(B, "B"));
+  if (A->dtype != B->dtype) return fail(GM_ERR_DTYPE, "A and B have different value types");
+  if (A->n_cols != B->n_rows) return fail(GM_ERR_DIM_MISMATCH, "A.n_cols != B.n_rows");
+  int n_dev = 0;
+  if (cudaGetDeviceCount(&n_dev) != cudaSuccess || n_dev == 0) {
+    cudaGetLastError();
+    return fail(GM_ERR_CUDA, "no CUDA device: this library has no CPU path");
+  }
+  gm_plan* p = new gm_plan();
+  p->A = *A;
+  p->B = *B;
+  p->sv = value_bytes(A->dtype);
+  p->smem_bytes = smem_bytes;
+  if (opts) p->opts = *opts;
+  p->plan_stream = static_cast<cudaStream_t>(cuda_stream);
+  const char* env = std::getenv("GM_TIMING");
+  p->times.enabled = env && env[0] == '1';
+  const int rc = build_plan(p, p->plan_stream);
+  if (rc != GM_OK) {
+    cudaStreamSynchronize(p->plan_stream);
+    gm_plan_destroy(p);
+    return rc;
+  }
+  *plan_out = p;
+  return GM_OK;
+}
+
+int gm_spgemm_plan(const gm_csr* A, const gm_csr* B, size_t smem_bytes, gm_plan** plan_out) {
+  return gm_spgemm_plan_ex(A, B, smem_bytes, nullptr, nullptr, plan_out);
+}
+
+int gm_spgemm_execute(gm_plan* plan, void* cuda_stream, gm_csr* C_out) {
+  if (!plan || !C_out) return fail(GM_ERR_INVALID_ARG, "plan or C_out is null");
+  std::memset(C_out, 0, sizeof(*C_out));
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  return plan->A.dtype == GM_F32 ? execute_t<float>(plan, st, C_out) : execute_t<double>(plan, st, C_out);
+}
+
+int gm_plan_get_info(const gm_plan* plan, gm_plan_info* out) {
+  if (!plan || !out) return fail(GM_ERR_INVALID_ARG, "null argument");
+  *out = plan->info;
+  return GM_OK;
+}
+
+int gm_exec_get_stats(const gm_plan* plan, gm_exec_stats* out) {
+  if (!plan || !out) return fail(GM_ERR_INVALID_ARG, "null argument");
+  *out = plan->stats;
+  return GM_OK;
+}
+
+int gm_plan_set_timing(gm_plan* plan, int enable) {
+  if (!plan) return fail(GM_ERR_INVALID_ARG, "null plan");
+  plan->times.enabled = enable != 0;
+  return GM_OK;
+}
+
+int gm_plan_get_row_products(const gm_plan* plan, int64_t* ip_out_device, void* cuda_stream) {
+  if (!plan || !ip_out_device) return fail(GM_ERR_INVALID_ARG, "null argument");
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  if (plan->A.n_rows > 0)
+    GM_CUDA(cudaMemcpyAsync(ip_out_device, plan->ip, static_cast<size_t>(plan->A.n_rows) * sizeof(int64_t),
+                            cudaMemcpyDeviceToDevice, st));
+  return GM_OK;
+}
+
+void gm_csr_free(gm_csr* C) {
+  if (!C) return;
+  dev_free(const_cast<int64_t*>(C->row_ptr), nullptr);
+  dev_free(const_cast<int32_t*>(C->col_idx), nullptr);
+  dev_free(const_cast<void*>(C->vals), nullptr);
+  std::memset(C, 0, sizeof(*C));
+}
+
+void gm_plan_destroy(gm_plan* plan) {
+  if (!plan) return;
+  for (auto& b : plan->owned) dev_free(b.p, plan->plan_stream);
+  delete plan;
+}
+
+int gm_spgemm_host(const gm_csr* A_host, const gm_csr* B_host, size_t smem_bytes, const gm_plan_opts* opts, gm_csr* C_host,
+                   int64_t c_capacity) {
+  GM_TRY(check_csr_arg(A_host, "A_host"));
+  GM_TRY(check_csr_arg(B_host, "B_host"));
+  if (!C_host || !C_host->row_ptr || c_capacity < 0) return fail(GM_ERR_INVALID_ARG, "C_host needs caller-owned buffers");
+  if (A_host->dtype != B_host->dtype) return fail(GM_ERR_DTYPE, "A and B have different value types");
+  const size_t sv = static_cast<size_t>(value_bytes(A_host->dtype));
+  cudaStream_t st = nullptr;
+  GM_CUDA(cudaStreamCreateWithFlags(&st, cudaStreamNonBlocking));
+  gm_csr dev[2];
+  std::vector<void*> tmp;
+  int rc = GM_OK;
+  auto upload = [&](const gm_csr* H, gm_csr* D) -> int {
+    *D = *H;
+    void* rp = dev_alloc(static_cast<size_t>(H->n_rows + 1) * 8, st);
+    void* ci = dev_alloc(static_cast<size_t>(H->nnz) * 4, st);
+    void* va = dev_alloc(static_cast<size_t>(H->nnz) * sv, st);
+    tmp.push_back(rp); tmp.push_back(ci); tmp.push_back(va);
+    if (!rp || !ci || !va) return fail(GM_ERR_OOM, "device allocation for an input failed");
+    GM_CUDA(cudaMemcpyAsync(rp, H->row_ptr, static_cast<size_t>(H->n_rows + 1) * 8, cudaMemcpyHostToDevice, st));
+    if (H->nnz > 0) {
+      GM_CUDA(cudaMemcpyAsync(ci, H->col_idx, static_cast<size_t>(H->nnz) * 4, cudaMemcpyHostToDevice, st));
+      GM_CUDA(cudaMemcpyAsync(va, H->vals, static_cast<size_t>(H->nnz) * sv, cudaMemcpyHostToDevice, st));
+    }
+    D->row_ptr = static_cast<const int64_t*>(rp);
+    D->col_idx = static_cast<const int32_t*>(ci);
+    D->vals = va;
+    return GM_OK;
+  };
+  gm_plan* plan = nullptr;
+  gm_csr C{};
+  rc = upload(A_host, &dev[0]);
+  if (rc == GM_OK) rc = upload(B_host, &dev[1]);
+  if (rc == GM_OK) rc = gm_spgemm_plan_ex(&dev[0], &dev[1], smem_bytes, opts, st, &plan);
+  if (rc == GM_OK) rc = gm_spgemm_execute(plan, st, &C);
+  if (rc == GM_OK) {
+    C_host->n_rows = C.n_rows;
+    C_host->n_cols = C.n_cols;
+    C_host->nnz = C.nnz;
+    C_host->dtype = C.dtype;
+    cudaError_t e = cudaMemcpyAsync(const_cast<int64_t*>(C_host->row_ptr), C.row_ptr, static_cast<size_t>(C.n_rows + 1) * 8,
+                                    cudaMemcpyDeviceToHost, st);
+    if (C.nnz > c_capacity) {
+      rc = fail(GM_ERR_CAPACITY, "C has " + std::to_string(C.nnz) + " entries, more than c_capacity");
+    } else if (C.nnz > 0 && e == cudaSuccess) {
+      if (!C_host->col_idx || !C_host->vals) {
+        rc = fail(GM_ERR_INVALID_ARG, "C_host->col_idx / vals are null");
+      } else {
+        e = cudaMemcpyAsync(const_cast<int32_t*>(C_host->col_idx), C.col_idx, static_cast<size_t>(C.nnz) * 4,
+                            cudaMemcpyDeviceToHost, st);
+        if (e == cudaSuccess)
+          e = cudaMemcpyAsync(const_cast<void*>(C_host->vals), C.vals, static_cast<size_t>(C.nnz) * sv,
+                              cudaMemcpyDeviceToHost, st);
+      }
+    }
+    cudaError_t e2 = cudaStreamSynchronize(st);
+    if (rc == GM_OK && (e != cudaSuccess || e2 != cudaSuccess)) rc = fail(GM_ERR_CUDA, "copy of C to the host failed");
+    dev_free(const_cast<int64_t*>(C.row_ptr), st);
+    dev_free(const_cast<int32_t*>(C.col_idx), st);
+    dev_free(const_cast<void*>(C.vals), st);
+  }
+  if (plan) {
+    plan->plan_stream = st;
+    gm_plan_destroy(plan);
+  }
+  for (void* q : tmp) dev_free(q, st);
+  cudaStreamSynchronize(st);
+  cudaStreamDestroy(st);
+  return rc;
+}
+
+const char* gm_status_string(int status) {
+  switch (status) {
+    case GM_OK: return "GM_OK";
+    case GM_ERR_INVALID_ARG: return "GM_ERR_INVALID_ARG";
+    case GM_ERR_DIM_MISMATCH: return "GM_ERR_DIM_MISMATCH";
+    case GM_ERR_DTYPE: return "GM_ERR_DTYPE";
+    case GM_ERR_BAD_CSR: return "GM_ERR_BAD_CSR";
+    case GM_ERR_OOM: return "GM_ERR_OOM";
+    case GM_ERR_CAPACITY: return "GM_ERR_CAPACITY";
+    case GM_ERR_CUDA: return "GM_ERR_CUDA";
+    case GM_ERR_TIMEOUT: return "GM_ERR_TIMEOUT";
+    case GM_ERR_UNSUPPORTED_SMEM: return "GM_ERR_UNSUPPORTED_SMEM";
+    case GM_ERR_INTERNAL: return "GM_ERR_INTERNAL";
+    default: return "GM_ERR_UNKNOWN";
+  }
+}
+
+const char* gm_last_error(void) { return g_last_error.c_str(); }
+
+}  // extern "C"

@@ -1,0 +1,81 @@
+// Shared device helpers: warp/block reductions and scans, search, error flag.
+#pragma once
+#include <cuda_runtime.h>
+
+#include <cstdint>
+
+namespace gm {
+
+using u32 = uint32_t;
+using u64 = unsigned long long;
+using i64 = int64_t;
+
+// Device-side status word: kernels never trap; they record the first problem here and skip the access.
+enum DevError : int {
+  kDevOk = 0,
+  kDevCapacity = 1,      // a write would have gone past the room reserved for C
+  kDevTableFull = 2,     // a light-row hash table overflowed (planner bug)
+  kDevBadChunk = 3,      // an element landed in a chunk that does not own its column
+};
+
+__device__ __forceinline__ void dev_set_error(int* flag, int code) { atomicCAS(flag, 0, code); }
+
+__device__ __forceinline__ u32 lanemask_lt() {
+  u32 m;
+  asm("mov.u32 %0, %%lanemask_lt;" : "=r"(m));
+  return m;
+}
+
+template <typename T>
+__device__ __forceinline__ T warp_sum(T v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  return v;
+}
+
+template <typename T>
+__device__ __forceinline__ T warp_inclusive_scan(T v) {
+  const int lane = threadIdx.x & 31;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    T n = __shfl_up_sync(0xffffffffu, v, o);
+    if (lane >= o) v += n;
+  }
+  return v;
+}
+
+// Exclusive scan of one value per thread over the whole block (blockDim.x a multiple of 32, at most 1024).
+// `warp_tmp` points to 33 T's of shared memory.  Returns the exclusive prefix; *total gets the block sum.
+// Contains two __syncthreads(); callers may reuse warp_tmp right after it returns only after another barrier.
+template <typename T>
+__device__ __forceinline__ T block_exclusive_scan(T v, T* warp_tmp, T* total) {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarps = (blockDim.x + 31) >> 5;
+  const T inc = warp_inclusive_scan(v);
+  if (lane == 31) warp_tmp[warp] = inc;
+  __syncthreads();
+  if (warp == 0) {
+    T w = lane < nwarps ? warp_tmp[lane] : T(0);
+    const T winc = warp_inclusive_scan(w);
+    warp_tmp[lane] = winc - w;
+    if (lane == 31) warp_tmp[32] = winc;
+  }
+  __syncthreads();
+  *total = warp_tmp[32];
+  return warp_tmp[warp] + inc - v;
+}
+
+// Largest index s in [lo, hi] with a[s] <= x, assuming a[lo] <= x and a non-decreasing.
+template <typename T, typename X>
+__device__ __forceinline__ i64 last_le(const T* __restrict__ a, i64 lo, i64 hi, X x) {
+  while (lo < hi) {
+    const i64 mid = lo + ((hi - lo + 1) >> 1);
+    if (static_cast<X>(a[mid]) <= x) lo = mid; else hi = mid - 1;
+  }
+  return lo;
+}
+
+__device__ __forceinline__ int clamp_rel(i64 v, int lo, int hi) {
+  return v < lo ? lo : (v > hi ? hi : static_cast<int>(v));
+}
+
+}  // namespace gm

@@ -1,0 +1,108 @@
+// K4 — expansion of the heavy rows' intermediate products (OuterProductKernel, Algorithm 4).
+//
+// The flattened product space of the heavy rows is cut into equal tiles, one per block (static,
+// locally computed partition, as in Algorithm 4's GroupRange).  Products are generated in row
+// order, so row h of the intermediate matrix owns the contiguous range [heavy_base[h],
+// heavy_base[h+1]) and no atomic reservation of output ranges is needed: segment s (one stored
+// entry of A scaled row of B) starts at seg_off[s], and product p of the tile is
+//     col = B.col[seg_bstart[s] + (p - seg_off[s])],  val = A.val[seg_j[s]] * B.val[...]
+// for the segment s that contains p (Eq. 3 with a division-free search).  Each warp walks a
+// contiguous part of the tile, so reads of B and writes of the staging buffer are coalesced runs.
+#pragma once
+#include "gm_common.cuh"
+
+namespace gm {
+
+constexpr int kExpandThreads = 256;
+constexpr int kExpandTile = 8192;     // products per block
+constexpr int kExpandSegCap = 1024;   // segments staged in shared memory; tiles with more take the slow path
+constexpr int kExpandUnroll = 4;
+
+template <typename V>
+__global__ void __launch_bounds__(kExpandThreads) k4_expand(
+    const i64* __restrict__ seg_off, const i64* __restrict__ seg_bstart, const i64* __restrict__ seg_j,
+    i64 seg_lo_all, i64 seg_hi_all,   // segments of this batch: [seg_lo_all, seg_hi_all)
+    const V* __restrict__ a_val, const int32_t* __restrict__ b_col, const V* __restrict__ b_val,
+    i64 elem0, i64 n_elems,           // first product of the batch (global heavy numbering), batch size
+    int32_t* __restrict__ x_col, V* __restrict__ x_val) {
+  __shared__ i64 s_range[2];
+  __shared__ int s_rel[kExpandSegCap + 1];
+  __shared__ i64 s_bstart[kExpandSegCap];
+  __shared__ V s_aval[kExpandSegCap];
+
+  const i64 t0 = static_cast<i64>(blockIdx.x) * kExpandTile;
+  const int tn = static_cast<int>(min(static_cast<i64>(kExpandTile), n_elems - t0));
+  const i64 p0 = elem0 + t0;  // global product index of the tile's first element
+  if (threadIdx.x < 2) {
+    const i64 p = threadIdx.x == 0 ? p0 : p0 + tn - 1;
+    s_range[threadIdx.x] = last_le(seg_off, seg_lo_all, seg_hi_all - 1, p);
+  }
+  __syncthreads();
+  const i64 s_lo = s_range[0];
+  const i64 n_seg = s_range[1] - s_lo + 1;
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  constexpr int kPerWarp = kExpandTile / (kExpandThreads / 32);
+  const int w0 = warp * kPerWarp;
+  const int w1 = min(tn, w0 + kPerWarp);
+
+  if (n_seg <= kExpandSegCap) {
+    for (int k = threadIdx.x; k <= n_seg; k += kExpandThreads) {
+      // start of segment k relative to the tile; > -2^31 because a row of B has < 2^31 entries
+      s_rel[k] = (k == n_seg) ? tn + 1 : static_cast<int>(max(seg_off[s_lo + k] - p0, static_cast<i64>(INT_MIN)));
+      if (k < n_seg) {
+        s_bstart[k] = seg_bstart[s_lo + k];
+        s_aval[k] = a_val[seg_j[s_lo + k]];
+      }
+    }
+    __syncthreads();
+    if (w0 >= w1) return;
+    // warp-uniform start: last segment whose start is <= w0 (zero-length segments are skipped by taking the last)
+    int cur = 0;
+    {
+      int lo = 0, hi = static_cast<int>(n_seg) - 1;
+      while (lo < hi) {
+        const int mid = lo + ((hi - lo + 1) >> 1);
+        if (s_rel[mid] <= w0) lo = mid; else hi = mid - 1;
+      }
+      cur = lo;
+    }
+    for (int q0 = w0; q0 < w1; q0 += 32 * kExpandUnroll) {
+      int32_t col[kExpandUnroll];
+      V val[kExpandUnroll], av[kExpandUnroll];
+#pragma unroll
+      for (int u = 0; u < kExpandUnroll; ++u) {
+        const int q = q0 + u * 32 + lane;
+        if (q < w1) {
+          int s = cur;
+          while (q >= s_rel[s + 1]) ++s;
+          const i64 src = s_bstart[s] + (q - s_rel[s]);
+          col[u] = b_col[src];
+          val[u] = b_val[src];
+          av[u] = s_aval[s];
+          cur = s;
+        }
+        cur = __shfl_sync(0xffffffffu, cur, 31);  // monotone: the last lane is furthest
+        // lanes past w1 keep their stale cur; lane 31 is only past w1 in the last step
+      }
+#pragma unroll
+      for (int u = 0; u < kExpandUnroll; ++u) {
+        const int q = q0 + u * 32 + lane;
+        if (q < w1) {
+          x_col[t0 + q] = col[u];
+          x_val[t0 + q] = av[u] * val[u];
+        }
+      }
+    }
+  } else {
+    // slow path: more segments than the shared table holds (very short rows of B): search per element
+    for (int q = threadIdx.x; q < tn; q += kExpandThreads) {
+      const i64 p = p0 + q;
+      const i64 s = last_le(seg_off, s_lo, s_range[1], p);
+      const i64 src = seg_bstart[s] + (p - seg_off[s]);
+      x_col[t0 + q] = b_col[src];
+      x_val[t0 + q] = a_val[seg_j[s]] * b_val[src];
+    }
+  }
+}
+
+}  // namespace gm

@@ -1,0 +1,208 @@
+// K5 — one level of the hierarchical multisplit (Histogram + MultisplitKernel, Algorithm 5).
+//
+// Input: the staging buffer X, whose elements are grouped by *parent* (a heavy row at level 0, a
+// chunk of the previous level afterwards); parent P owns [parent_off[P], parent_off[P+1]).
+// Output: Y, where the elements of every parent are regrouped into F children by
+//     child = (col >> shift) & (F - 1)
+// and child (P, c) owns [child_off[P*F+c], child_off[P*F+c+1]) — the children tile their parent's
+// range in order, so child_off is the plain exclusive scan of the (parent, child) count matrix.
+//
+// Both kernels use the same static partition of the flattened element space into tiles (GroupRange
+// of Algorithm 5) and the same per-tile binning: bin = parent_in_tile * F + child, counted with a
+// warp-level match (lanes that hit the same bin elect one leader, which adds the group's size with
+// one shared-memory atomic and hands each member its rank).
+//   k5_histogram : adds the tile's bin counts to the global count matrix.
+//   k5_multisplit: reserves the tile's share of every child's output range with one global atomic
+//                  per non-empty bin (the cursor array starts as a copy of child_off), permutes
+//                  the tile by bin in shared memory, and writes it out bin after bin, so each
+//                  child receives a contiguous, coalesced run.
+// A tile whose bins do not fit the shared table (very many tiny parents) falls back to one global
+// atomic per element.
+#pragma once
+#include "gm_common.cuh"
+
+namespace gm {
+
+constexpr int kSplitThreads = 512;
+constexpr int kSplitItems = 16;
+constexpr int kSplitTile = kSplitThreads * kSplitItems;  // 8192 elements per block
+constexpr int kSplitBinCap = 2048;                       // bins (parent, child) per tile in shared memory
+constexpr int kSplitParentCap = 256;                     // parents per tile on the fast path
+
+template <typename V>
+constexpr size_t split_smem_bytes(bool multisplit) {
+  // bins + parent offsets + parent starts (+ permuted columns and values)
+  size_t b = kSplitBinCap * 4 + (kSplitParentCap + 1) * 4 + kSplitParentCap * 4 + 64;
+  if (multisplit) b += static_cast<size_t>(kSplitTile) * (4 + sizeof(V));
+  return b;
+}
+
+struct SplitTileInfo {
+  i64 p_lo;   // first parent touching the tile
+  int n_par;  // parents touching the tile (including empty ones in between)
+};
+
+template <typename V, bool MULTISPLIT>
+__global__ void __launch_bounds__(kSplitThreads, 2) k5_level(
+    const int32_t* __restrict__ x_col, const V* __restrict__ x_val, i64 n_elems,
+    const i64* __restrict__ parent_off, i64 n_parents, int F, int shift,
+    u32* __restrict__ counts,     // histogram: (n_parents * F) counters, zero-initialised
+    u64* __restrict__ cursor,     // multisplit: (n_parents * F) write cursors, start = child_off
+    int32_t* __restrict__ y_col, V* __restrict__ y_val) {
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  u32* s_bin = reinterpret_cast<u32*>(smem_raw);                     // kSplitBinCap: counts -> starts -> deltas
+  int* s_poff = reinterpret_cast<int*>(s_bin + kSplitBinCap);        // kSplitParentCap + 1: parent starts rel. to tile
+  int* s_pstart = s_poff + kSplitParentCap + 1;                      // kSplitParentCap: first permuted slot of a parent
+  V* s_val = reinterpret_cast<V*>(s_pstart + kSplitParentCap + 15);  // aligned below
+  s_val = reinterpret_cast<V*>((reinterpret_cast<uintptr_t>(s_val)) & ~uintptr_t{15});
+  int32_t* s_col = reinterpret_cast<int32_t*>(s_val + kSplitTile);
+  __shared__ i64 s_range[2];
+  __shared__ u32 s_scan[33];
+
+  const i64 t0 = static_cast<i64>(blockIdx.x) * kSplitTile;
+  const int tn = static_cast<int>(min(static_cast<i64>(kSplitTile), n_elems - t0));
+  const int tid = threadIdx.x, lane = tid & 31;
+  if (tid < 2) s_range[tid] = last_le(parent_off, 0, n_parents - 1, tid == 0 ? t0 : t0 + tn - 1);
+  __syncthreads();
+  const i64 p_lo = s_range[0];
+  const i64 n_par64 = s_range[1] - p_lo + 1;
+  const u32 fmask = static_cast<u32>(F - 1);
+
+  if (n_par64 > kSplitParentCap || n_par64 * F > kSplitBinCap) {
+    // ---- slow path: one global atomic per element
+    for (int q = tid; q < tn; q += kSplitThreads) {
+      const i64 p = t0 + q;
+      const i64 par = last_le(parent_off, p_lo, s_range[1], p);
+      const int32_t c = x_col[p];
+      const i64 gbin = par * F + ((static_cast<u32>(c) >> shift) & fmask);
+      if (MULTISPLIT) {
+        const u64 dst = atomicAdd(&cursor[gbin], 1ull);
+        y_col[dst] = c;
+        y_val[dst] = x_val[p];
+      } else {
+        atomicAdd(&counts[gbin], 1u);
+      }
+    }
+    return;
+  }
+  const int n_par = static_cast<int>(n_par64);
+  const int n_bins = n_par * F;
+  for (int b = tid; b < n_bins; b += kSplitThreads) s_bin[b] = 0;
+  for (int k = tid; k <= n_par; k += kSplitThreads)
+    s_poff[k] = (k == n_par) ? tn + 1 : clamp_rel(parent_off[p_lo + k] - t0, -1, tn + 1);
+  __syncthreads();
+
+  // ---- local histogram with warp-level match; every element learns its rank inside its bin
+  int32_t col[kSplitItems];
+  u32 rank_bin[kSplitItems];  // (rank << 11) | bin
+  static_assert(kSplitBinCap <= 2048 && kSplitTile <= (1 << 21), "rank/bin packing");
+#pragma unroll
+  for (int k = 0; k < kSplitItems; ++k) {
+    const int q = k * kSplitThreads + tid;
+    u32 bin = 0xffffffffu;
+    if (q < tn) {
+      col[k] = x_col[t0 + q];
+      int par = 0;
+      if (n_par > 1) {
+        int lo = 0, hi = n_par - 1;
+        while (lo < hi) {
+          const int mid = lo + ((hi - lo + 1) >> 1);
+          if (s_poff[mid] <= q) lo = mid; else hi = mid - 1;
+        }
+        par = lo;
+      }
+      bin = static_cast<u32>(par * F) + ((static_cast<u32>(col[k]) >> shift) & fmask);
+    }
+    const u32 peers = __match_any_sync(0xffffffffu, bin);
+    const int leader = __ffs(peers) - 1;
+    u32 old = 0;
+    if (lane == leader && bin != 0xffffffffu) old = atomicAdd(&s_bin[bin], static_cast<u32>(__popc(peers)));
+    old = __shfl_sync(0xffffffffu, old, leader);
+    rank_bin[k] = ((old + __popc(peers & lanemask_lt())) << 11) | (bin & 2047u);
+  }
+  __syncthreads();
+
+  // ---- scan of the bin counts; global update (histogram) or range reservation (multisplit)
+  constexpr int kBinsPerThread = kSplitBinCap / kSplitThreads;
+  u32 cnt[kBinsPerThread];
+  u32 sum = 0;
+#pragma unroll
+  for (int k = 0; k < kBinsPerThread; ++k) {
+    const int b = tid * kBinsPerThread + k;
+    cnt[k] = b < n_bins ? s_bin[b] : 0u;
+    sum += cnt[k];
+  }
+  const i64 gbin0 = p_lo * F;
+  if (!MULTISPLIT) {
+#pragma unroll
+    for (int k = 0; k < kBinsPerThread; ++k) {
+      const int b = tid * kBinsPerThread + k;
+      if (cnt[k]) atomicAdd(&counts[gbin0 + b], cnt[k]);
+    }
+    return;
+  }
+  u32 total;
+  u32 start = block_exclusive_scan(sum, s_scan, &total);
+  u32 delta[kBinsPerThread];
+#pragma unroll
+  for (int k = 0; k < kBinsPerThread; ++k) {
+    const int b = tid * kBinsPerThread + k;
+    if (b < n_bins) {
+      s_bin[b] = start;  // own slots only: nobody else reads them before the barrier
+      if ((b % F) == 0) s_pstart[b / F] = static_cast<int>(start);
+      delta[k] = cnt[k] ? static_cast<u32>(atomicAdd(&cursor[gbin0 + b], static_cast<u64>(cnt[k]))) - start : 0u;
+    }
+    start += cnt[k];
+  }
+  __syncthreads();
+
+  // ---- permute into shared memory (the irregular part stays on chip)
+#pragma unroll
+  for (int h = 0; h < kSplitItems; h += 8) {
+    V v[8];
+#pragma unroll
+    for (int k = 0; k < 8; ++k) {
+      const int q = (h + k) * kSplitThreads + tid;
+      if (q < tn) v[k] = x_val[t0 + q];
+    }
+#pragma unroll
+    for (int k = 0; k < 8; ++k) {
+      const int q = (h + k) * kSplitThreads + tid;
+      if (q < tn) {
+        const u32 rb = rank_bin[h + k];
+        const u32 dst = s_bin[rb & 2047u] + (rb >> 11);
+        s_col[dst] = col[h + k];
+        s_val[dst] = v[k];
+      }
+    }
+  }
+  __syncthreads();
+#pragma unroll
+  for (int k = 0; k < kBinsPerThread; ++k) {
+    const int b = tid * kBinsPerThread + k;
+    if (b < n_bins) s_bin[b] = delta[k];  // global position of slot s in bin b is s + delta[b] (mod 2^32 within the batch)
+  }
+  __syncthreads();
+
+  // ---- coalesced write: slot s belongs to the bin recomputed from its column and its parent
+  const u64 hi_base = 0;  // batch-relative positions fit 32 bits (checked by the planner)
+  (void)hi_base;
+  for (int s = tid; s < tn; s += kSplitThreads) {
+    const int32_t c = s_col[s];
+    int par = 0;
+    if (n_par > 1) {
+      int lo = 0, hi = n_par - 1;
+      while (lo < hi) {
+        const int mid = lo + ((hi - lo + 1) >> 1);
+        if (s_pstart[mid] <= s) lo = mid; else hi = mid - 1;
+      }
+      par = lo;
+    }
+    const u32 bin = static_cast<u32>(par * F) + ((static_cast<u32>(c) >> shift) & fmask);
+    const u32 dst = static_cast<u32>(s) + s_bin[bin];
+    y_col[dst] = c;
+    y_val[dst] = s_val[s];
+  }
+}
+
+}  // namespace gm

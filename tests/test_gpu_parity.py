@@ -1,0 +1,214 @@
+"""GPU parity tests: the CUDA path, called through the C ABI, against the CPU oracle on the same
+seeded inputs.  Structure (row_ptr, col_idx) bit-exact; values within tau * sum|a*b| with
+tau = 1e-5 (fp32) / 1e-12 (fp64)."""
+import numpy as np
+import pytest
+import torch
+
+import gen
+import oracle
+from helpers import csr_from_pattern, random_csr
+from parity import check_product, run_gpu, compare_rows
+
+pytestmark = pytest.mark.gpu
+
+
+def test_row_analysis_matches_definition():
+    import paper_2607_22866_b200 as gm
+    A, B, _ = gen.config_inputs(4, shrink=6)
+    dA, dB = gm.DeviceCSR.from_host(A), gm.DeviceCSR.from_host(B)
+    plan = gm.spgemm_plan(dA, dB)
+    ip = plan.row_products().cpu().numpy()
+    ref = oracle.row_products(A, B)
+    assert np.array_equal(ip, ref)
+    info = plan.info()
+    assert info.products_total == ref.sum() and info.products_max_row == ref.max()
+    assert info.rows_empty == int((ref == 0).sum())
+    assert info.c_nnz_upper == int(np.minimum(ref, B.n_cols).sum())
+    plan.destroy()
+
+
+def test_config0_er_all_light():
+    A, B, _ = gen.config_inputs(0)
+    C, info, stats = check_product(A, B)
+    assert info.rows_heavy == 0 and info.rows_light == 4096 and info.products_total == 262144
+
+
+@pytest.mark.parametrize("shrink", [4, 0])
+def test_config1_laplacian_bit_exact(shrink):
+    A, B, _ = gen.config_inputs(1, shrink=shrink)
+    C, info, stats = check_product(A, B)
+    N = 1024 >> shrink
+    assert C.nnz == 13 * N * N - 20 * N + 4
+    # small integers: fp64 sums are exact whatever the order
+    ref = oracle.spgemm(A, B)
+    assert np.array_equal(C.val.cpu().numpy(), ref.val)
+
+
+@pytest.mark.parametrize("cfg,shrink", [(2, 8), (2, 6), (3, 8), (4, 6)])
+def test_scaled_down_configs_default_plan(cfg, shrink):
+    A, B, _ = gen.config_inputs(cfg, shrink=shrink)
+    check_product(A, B)
+
+
+@pytest.mark.parametrize("dtype", [np.float32, np.float64])
+@pytest.mark.parametrize("levels", [0, 1, 2, 3])
+def test_forced_levels_give_identical_structure(dtype, levels):
+    A = gen.rmat(12, 16, seed=3, dtype=dtype)
+    width = {0: 4096, 1: 1024, 2: 256, 3: 64}[levels]
+    fan = {0: 0, 1: 4, 2: 4, 3: 4}[levels]
+    C, info, stats = check_product(A, A, tau=256, chunk_width=width, max_fanout=fan)
+    assert info.params.n_levels == levels
+    assert info.rows_heavy > 100 and stats.final_chunks == info.rows_heavy * info.params.chunks_required
+
+
+@pytest.mark.parametrize("dtype", [np.float32, np.float64])
+def test_many_batches_append_in_row_order(dtype):
+    A = gen.rmat(12, 16, seed=5, dtype=dtype)
+    ip = oracle.row_products(A, A)
+    # staging barely larger than the biggest row: dozens of batches, some holding a single row
+    C, info, stats = check_product(A, A, tau=128, chunk_width=512, max_fanout=8, stage_elems=int(ip.max()) + 1000)
+    assert info.n_batches > 8
+    assert stats.c_capacity >= C.nnz
+
+
+def test_capacity_error_is_reported_not_faulted():
+    import paper_2607_22866_b200 as gm
+    A = gen.rmat(11, 16, seed=6, dtype=np.float32)
+    ip = oracle.row_products(A, A)
+    with pytest.raises(gm.GmError) as ei:
+        run_gpu(A, A, tau=128, chunk_width=512, stage_elems=int(ip.max()) + 100, c_capacity=1000)
+    assert ei.value.status == -6
+    with pytest.raises(gm.GmError) as ei:
+        run_gpu(A, A, tau=128, stage_elems=int(ip.max()) - 1)   # a row is never split across batches
+    assert ei.value.status == -6
+    # the context is still usable
+    check_product(A, A, tau=128, chunk_width=512)
+
+
+@pytest.mark.parametrize("smem", [49152, 101376, 232448])
+def test_smem_budget_sweep(smem):
+    A = gen.rmat(13, 16, seed=7, dtype=np.float32)
+    C, info, stats = check_product(A, A, smem_bytes=smem)
+    assert info.params.tau <= 8192
+
+
+@pytest.mark.parametrize("dtype", [np.float32, np.float64])
+def test_light_heavy_boundary_and_degenerate_rows(dtype):
+    rng = np.random.default_rng(3)
+    n, m = 300, 1000
+    # B: row 0 has a single entry (column 999), row 1 is dense, row 2 is empty, the rest random
+    patB = rng.random((n, m)) < 0.05
+    patB[0, :] = False; patB[0, 999] = True
+    patB[1, :] = True
+    patB[2, :] = False
+    B = csr_from_pattern(patB, rng.uniform(-1, 1, patB.shape), dtype)
+    patA = rng.random((64, n)) < 0.03
+    patA[5, :] = False; patA[5, 0] = True                  # one product
+    patA[6, :] = False; patA[6, [0, 2]] = True             # references an empty row of B
+    patA[7, :] = False                                      # empty row between heavy rows
+    patA[8, :] = True                                       # very heavy row (hits the dense row)
+    patA[9, :] = False; patA[9, 1] = True                  # exactly m products, all distinct columns
+    A = csr_from_pattern(patA, rng.uniform(-1, 1, patA.shape), dtype)
+    ip = oracle.row_products(A, B)
+    for tau in (int(ip[9]), int(ip[9]) - 1, 1, 40):        # IP_i == tau is light, tau + 1 is heavy
+        C, info, stats = check_product(A, B, tau=tau, chunk_width=128, max_fanout=2)
+        assert info.rows_heavy == int((ip > tau).sum())
+
+
+def test_heavy_row_whose_products_hit_one_column_or_one_chunk():
+    dtype = np.float32
+    n = 600
+    # every row of B is the same single entry in column 77 => a heavy row of A gives ONE entry of C
+    patB = np.zeros((n, 4096), bool); patB[:, 77] = True
+    rng = np.random.default_rng(5)
+    B = csr_from_pattern(patB, rng.uniform(-1, 1, patB.shape), dtype)
+    patA = np.zeros((4, n), bool); patA[1, :] = True; patA[3, :500] = True
+    A = csr_from_pattern(patA, rng.uniform(-1, 1, patA.shape), dtype)
+    C, info, stats = check_product(A, B, tau=64, chunk_width=256, max_fanout=4)
+    assert info.rows_heavy == 2 and C.nnz == 2
+    # exactly one product per chunk: B rows are single entries at columns c*W
+    patB2 = np.zeros((16, 4096), bool)
+    for k in range(16):
+        patB2[k, k * 256] = True
+    B2 = csr_from_pattern(patB2, np.ones(patB2.shape), dtype)
+    A2 = csr_from_pattern(np.ones((2, 16), bool), rng.uniform(-1, 1, (2, 16)), dtype)
+    check_product(A2, B2, tau=8, chunk_width=256, max_fanout=4)
+
+
+@pytest.mark.parametrize("c_cols", [1, 31, 255, 256, 257, 100003])
+def test_column_counts_that_are_not_chunk_multiples(c_cols):
+    rng = np.random.default_rng(c_cols)
+    k = 200
+    dens = min(0.5, 60.0 / c_cols) if c_cols > 1 else 1.0
+    B = random_csr(rng, k, c_cols, dens, np.float64)
+    A = random_csr(rng, 50, k, 0.3, np.float64)
+    check_product(A, B, tau=16, chunk_width=256 if c_cols > 256 else 32, max_fanout=4)
+
+
+def test_empty_operands():
+    for shape_a, shape_b in [((0, 5), (5, 7)), ((4, 0), (0, 7)), ((4, 5), (5, 0)), ((3, 3), (3, 3))]:
+        A = csr_from_pattern(np.zeros(shape_a, bool), np.zeros(shape_a), np.float32)
+        B = csr_from_pattern(np.zeros(shape_b, bool), np.zeros(shape_b), np.float32)
+        C, info, stats = run_gpu(A, B)
+        assert C.nnz == 0 and C.row_ptr.numel() == shape_a[0] + 1 and int(C.row_ptr.abs().sum()) == 0
+
+
+def test_argument_errors():
+    import paper_2607_22866_b200 as gm
+    A = gen.erdos_renyi_k(64, 4, seed=1, dtype=np.float32)
+    B = gen.erdos_renyi_k(32, 4, seed=1, dtype=np.float32)
+    with pytest.raises(gm.GmError) as ei:
+        run_gpu(A, B)
+    assert ei.value.status == -2
+    A64 = gen.erdos_renyi_k(64, 4, seed=1, dtype=np.float64)
+    with pytest.raises(gm.GmError) as ei:
+        gm.spgemm(gm.DeviceCSR.from_host(A), gm.DeviceCSR.from_host(A64))
+    assert ei.value.status == -3
+    with pytest.raises(gm.GmError) as ei:
+        run_gpu(A, A, smem_bytes=1 << 19)
+    assert ei.value.status == -9
+    bad = gen.erdos_renyi_k(64, 4, seed=1, dtype=np.float32)
+    bad.col[1] = bad.col[0]        # duplicate column in row 0
+    with pytest.raises(gm.GmError) as ei:
+        run_gpu(bad, A, validate_inputs=1)
+    assert ei.value.status == -4
+
+
+def test_two_runs_same_structure_values_close():
+    A = gen.rmat(12, 16, seed=9, dtype=np.float32)
+    C1, _, _ = run_gpu(A, A, tau=256, chunk_width=1024, max_fanout=4)
+    C2, _, _ = run_gpu(A, A, tau=256, chunk_width=1024, max_fanout=4)
+    assert torch.equal(C1.row_ptr, C2.row_ptr) and torch.equal(C1.col, C2.col)
+    ref = oracle.spgemm(A, A)
+    d = (C1.val.double() - C2.val.double()).abs().cpu().numpy()
+    assert np.all(d <= 2e-5 * ref.abs)
+
+
+def test_plan_reuse_with_new_values():
+    import paper_2607_22866_b200 as gm
+    A = gen.rmat(11, 16, seed=2, dtype=np.float64)
+    dA = gm.DeviceCSR.from_host(A)
+    plan = gm.spgemm_plan(dA, dA, opts=None)
+    C1 = gm.spgemm_execute(plan)
+    compare_rows(C1, oracle.spgemm(A, A), np.float64)
+    dA.val.mul_(-0.5)
+    A.val[:] = A.val * -0.5
+    C2 = gm.spgemm_execute(plan)
+    compare_rows(C2, oracle.spgemm(A, A), np.float64)
+    plan.destroy()
+
+
+def test_host_entry_point():
+    import paper_2607_22866_b200 as gm
+    A, B, _ = gen.config_inputs(4, shrink=7)
+    ref = oracle.spgemm(A, B)
+    rp = np.empty(A.n_rows + 1, np.int64)
+    col = np.empty(ref.nnz + 10, np.int32)
+    val = np.empty(ref.nnz + 10, np.float32)
+    nnz = gm.spgemm_host(A, B, rp, col, val)
+    assert nnz == ref.nnz and np.array_equal(rp, ref.row_ptr) and np.array_equal(col[:nnz], ref.col)
+    assert np.all(np.abs(val[:nnz].astype(np.float64) - ref.val) <= 1e-5 * ref.abs)
+    with pytest.raises(gm.GmError) as ei:
+        gm.spgemm_host(A, B, rp, col[:5], val[:5])
+    assert ei.value.status == -6
