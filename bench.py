@@ -1,0 +1,360 @@
+#!/usr/bin/env python
+"""Benchmark of the SpGEMM hot path (plan + execute = every step of Algorithm 3) on synthetic inputs.
+
+    python bench.py --gpus 1 --steps 5 --warmup 3            # CUDA library, default workload
+    python bench.py --impl reference --steps 2 --warmup 1    # CPU oracle on a bounded row sample
+
+One "step" is one whole product C = A*B: row analysis, planning, light rows, and for the heavy rows
+expansion, every multisplit level and the chunk accumulation, with A and B resident in HBM.  The
+metric is SpGEMM GFLOP/s = 2 * intermediate products / time.  The line also carries the roofline
+of the dominant kernel, the oracle timed on the host cores, and an end-to-end number measured
+through the host-buffer entry point (copies inside the timed region).
+
+Multi-GPU: the path does not shard in this build ("replicas only"): with --gpus N every rank runs
+the same product on its own GPU, no collective touches the data path.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import tempfile
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import gen  # noqa: E402
+
+SMEM_BYTES = 232448
+DEFAULT_CONFIG = 2  # R-MAT scale 20, edge factor 16, fp32: the largest fp32 power-law product
+
+
+def _peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    return 6650.0, "fallback"
+
+
+class ClockSampler:
+    """nvidia-smi sampling of SM clocks and throttle reasons during the timed region."""
+    FIELDS = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+              "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+              "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.gpu_index, self.proc, self.path = gpu_index, None, None
+
+    def start(self):
+        try:
+            fd, self.path = tempfile.mkstemp(suffix=".csv")
+            os.close(fd)
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits", "-lms", "200",
+                 "-i", str(self.gpu_index)], stdout=open(self.path, "w"), stderr=subprocess.DEVNULL)
+        except Exception:
+            self.proc = None
+
+    def stop(self) -> dict:
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": []}
+        if self.proc is None:
+            return out
+        time.sleep(0.25)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        try:
+            for line in open(self.path):
+                f = [x.strip() for x in line.split(",")]
+                if len(f) < 9:
+                    continue
+                sm.append(float(f[1])), mx.append(float(f[2]))
+                for name, v in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), f[5:9]):
+                    if v.lower().startswith("active"):
+                        reasons.add(name)
+            os.unlink(self.path)
+        except Exception:
+            pass
+        if sm:
+            out.update(sm_mhz=statistics.median(sm), sm_max_mhz=max(mx), reasons=sorted(reasons), samples=len(sm))
+        return out
+
+
+def _row_sample(n_rows: int, blocks: int, frac: float):
+    """`blocks` evenly spaced contiguous row ranges that together cover `frac` of the rows."""
+    blocks = max(1, min(blocks, n_rows))
+    width = max(1, int(n_rows * frac / blocks))
+    starts = np.linspace(0, max(n_rows - width, 0), blocks).astype(np.int64)
+    return [(int(s), int(min(n_rows, s + width))) for s in starts]
+
+
+def oracle_timed(A, B, budget_s: float = 15.0):
+    """Times the CPU oracle (as it stands) on a bounded, evenly spread sample of row blocks.  Returns
+    (gflops, cores, description, seconds, products)."""
+    import oracle
+
+    ip = oracle.row_products(A, B)
+    total = int(ip.sum())
+    # calibrate on a small sample, then size the real one for roughly `budget_s`
+    cal = _row_sample(A.n_rows, 16, 0.002)
+    t = time.perf_counter()
+    threads = 1
+    for r0, r1 in cal:
+        threads = oracle.spgemm(A, B, r0, r1).threads
+    dt = max(time.perf_counter() - t, 1e-4)
+    cal_products = sum(int(ip[r0:r1].sum()) for r0, r1 in cal)
+    rate = max(cal_products, 1) / dt
+    frac = min(1.0, max(0.004, budget_s * rate / max(total, 1)))
+    blocks = _row_sample(A.n_rows, 64, frac)
+    products = sum(int(ip[r0:r1].sum()) for r0, r1 in blocks)
+    t = time.perf_counter()
+    for r0, r1 in blocks:
+        oracle.spgemm(A, B, r0, r1)
+    dt = time.perf_counter() - t
+    desc = (f"{len(blocks)} evenly spaced row blocks = {100.0 * sum(b - a for a, b in blocks) / max(A.n_rows, 1):.2f}% of rows, "
+            f"{products} of {total} products, {dt:.1f} s")
+    return 2.0 * products / dt / 1e9, threads, desc, dt, products
+
+
+def kernel_table(info, stats_avg, sv, nnz_b, n_light_entries_a):
+    """Algorithmic (minimum) bytes per step for every kernel of the path, with its measured time."""
+    se = 4 + sv
+    e = info.products_heavy
+    p = info.params
+    rows_h = info.rows_heavy
+    L = p.n_levels
+    nnz_c, nnz_ch = stats_avg["c_nnz"], stats_avg["c_nnz_heavy"]
+    chunks = stats_avg["final_chunks"]
+    parents = [rows_h]
+    for l in range(L):
+        parents.append(parents[-1] * p.fanout[l])
+    hist = sum(4 * e + 8 * (parents[l] + 1) + 4 * parents[l + 1] for l in range(L))
+    split = sum(2 * se * e + 8 * (parents[l] + 1) + 8 * parents[l + 1] for l in range(L))
+    tbl = {
+        "k3_light_symbolic": (4 * n_light_entries_a + 8 * info.rows_light + 4 * nnz_b, stats_avg["ms_light_symbolic"]),
+        "k3_light_numeric": (se * n_light_entries_a + se * nnz_b + se * (nnz_c - nnz_ch), stats_avg["ms_light_numeric"]),
+        "k4_expand": (se * e + se * nnz_b + 24 * info.nnz_a_heavy, stats_avg["ms_expand"]),
+        "k5a_histogram": (hist, stats_avg["ms_histogram"]),
+        "k5b_multisplit": (split, stats_avg["ms_multisplit"]),
+        "k6_accumulate_symbolic": (4 * e + 12 * chunks, stats_avg["ms_acc_symbolic"]),
+        "k6_accumulate_numeric": (se * e + se * nnz_ch + 24 * chunks, stats_avg["ms_acc_numeric"]),
+    }
+    return {k: {"bytes": int(b), "ms": float(ms), "gbs": (b / ms / 1e6 if ms > 0 else 0.0)} for k, (b, ms) in tbl.items()}
+
+
+def run_reference(args, A, B, desc):
+    vals, used = [], 1
+    sample = ""
+    for i in range(args.warmup + args.steps):
+        gf, used, sample, dt, products = oracle_timed(A, B, budget_s=args.cpu_budget)
+        if i >= args.warmup:
+            vals.append((gf, dt))
+    value = statistics.mean(v for v, _ in vals)
+    ms = statistics.mean(d for _, d in vals) * 1e3
+    line = {
+        "impl": "reference", "metric": "spgemm_gflops", "value": value, "unit": "GFLOP/s", "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f32" if A.val.dtype == np.float32 else "f64", "data": "synthetic",
+        "config": {"workload": gen.CONFIG_NAMES[args.config], "description": desc,
+                   "note": "CPU oracle (plain Gustavson) timed on a bounded row sample per step"},
+        "cpu_baseline": {"value": value, "unit": "GFLOP/s", "cores": used, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": "GFLOP/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=5)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--config", type=int, default=DEFAULT_CONFIG, help="index into the five workloads (0..4)")
+    ap.add_argument("--shrink", type=int, default=0, help="scale the workload down by 2**shrink (debugging)")
+    ap.add_argument("--cpu-budget", type=float, default=15.0, help="seconds of oracle time for the CPU baseline")
+    ap.add_argument("--e2e-steps", type=int, default=2)
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 1)
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+
+    if args.impl == "reference":
+        if rank != 0:
+            return
+        A, B, desc = gen.config_inputs(args.config, args.shrink)
+        run_reference(args, A, B, desc)
+        return
+
+    import torch
+    import torch.distributed as dist
+
+    import paper_2607_22866_b200 as gm
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the library has no CPU path")
+    torch.cuda.set_device(local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+
+    A, B, desc = gen.config_inputs(args.config, args.shrink)
+    sv = A.val.dtype.itemsize
+    dA = gm.DeviceCSR.from_host(A)
+    dB = dA if B is A else gm.DeviceCSR.from_host(B)
+    opts = gm.PlanOpts()
+
+    def step(timing: bool):
+        plan = gm.spgemm_plan(dA, dB, SMEM_BYTES, opts)
+        if timing:
+            plan.set_timing(True)
+        C = gm.spgemm_execute(plan)
+        info, st = plan.info(), plan.stats()
+        nnz = C.nnz
+        del C
+        plan.destroy()
+        return info, st, nnz
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(args.warmup):
+        info, st, nnz = step(False)
+    barrier()
+    sampler = ClockSampler(local_rank)
+    sampler.start()
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    ev0.record()
+    launches = 0
+    stats_sum: dict[str, float] = {}
+    for _ in range(args.steps):
+        info, st, nnz = step(True)
+        launches += int(info.launches + st.launches)
+        for name, _t in st._fields_:
+            if name != "reserved":
+                stats_sum[name] = stats_sum.get(name, 0.0) + float(getattr(st, name))
+    ev1.record()
+    barrier()
+    clocks = sampler.stop()
+    ms_total = ev0.elapsed_time(ev1)
+    t = torch.tensor([ms_total], device="cuda", dtype=torch.float64)
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    ms_step = float(t.item()) / args.steps
+    products = int(info.products_total)
+    value = world * 2.0 * products / (ms_step * 1e-3) / 1e9
+    stats_avg = {k: v / args.steps for k, v in stats_sum.items()}
+
+    # ---- roofline of the dominant kernel (times: CUDA events recorded by the library on the execute stream)
+    peak, peak_kind = _peaks()
+    a_len = np.diff(A.row_ptr)
+    tau = info.params.tau
+    plan = gm.spgemm_plan(dA, dB, SMEM_BYTES, opts)   # untimed: the row analysis feeds the byte model
+    ip_dev = plan.row_products().cpu().numpy()
+    plan.destroy()
+    n_light_entries_a = int(a_len[ip_dev <= tau].sum())
+    kt = kernel_table(info, stats_avg, sv, B.nnz, n_light_entries_a)
+    dom = max(kt, key=lambda k: kt[k]["ms"])
+    n_b = max(int(info.n_batches), 1)
+    per_launch = {"k4_expand": n_b, "k5a_histogram": n_b * max(info.params.n_levels, 1),
+                  "k5b_multisplit": n_b * max(info.params.n_levels, 1), "k6_accumulate_symbolic": n_b,
+                  "k6_accumulate_numeric": n_b}.get(dom, 1)
+    roofline = {"kernel": dom, "bound": "hbm", "achieved": kt[dom]["gbs"], "peak": peak, "unit": "GB/s",
+                "frac": kt[dom]["gbs"] / peak, "peak_kind": f"of {peak_kind}", "traffic": None,
+                "bytes_per_launch": kt[dom]["bytes"] / per_launch, "ms_per_launch": kt[dom]["ms"] / per_launch,
+                "launches_per_step": per_launch}
+
+    line = {
+        "metric": "spgemm_gflops", "value": value, "unit": "GFLOP/s", "n_gpus": world, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "f32" if sv == 4 else "f64", "data": "synthetic",
+        "config": {"workload": gen.CONFIG_NAMES[args.config] + (f"_shrink{args.shrink}" if args.shrink else ""),
+                   "description": desc, "parallelism": "replicas only" if world > 1 else "1 gpu",
+                   "l2": "inputs, staging and C are far larger than L2 (126 MB); no flush needed",
+                   "products": products, "products_heavy": int(info.products_heavy), "nnz_c": int(nnz),
+                   "rows_heavy": int(info.rows_heavy), "tau": int(tau), "chunk_width": int(info.params.chunk_width),
+                   "levels": info.params.levels(), "batches": int(info.n_batches), "smem_bytes": SMEM_BYTES,
+                   "step": "gm_spgemm_plan + gm_spgemm_execute (C freed after each step)"},
+        "roofline": roofline, "kernels": kt, "clocks": clocks, "gpu_launches": launches,
+    }
+
+    if rank == 0 and not args.no_e2e:
+        line["e2e"] = e2e_leg(gm, torch, A, B, int(nnz), products, args.e2e_steps)
+    if rank == 0 and not args.no_cpu_baseline:
+        gf, cores, sample, _dt, _p = oracle_timed(A, B, budget_s=args.cpu_budget)
+        line["cpu_baseline"] = {"value": gf, "unit": "GFLOP/s", "cores": cores, "kind": "oracle", "sample": sample}
+    if world > 1:
+        dist.barrier()
+        dist.destroy_process_group()
+    if rank == 0:
+        print(json.dumps(line))
+
+
+def e2e_leg(gm, torch, A, B, nnz, products, steps):
+    """Same product through gm_spgemm_host: A and B start in pinned host memory, C ends in pinned host
+    memory; the copies are inside the timed region."""
+    sv = A.val.dtype.itemsize
+
+    def pinned(arr):
+        t = torch.from_numpy(arr)
+        try:
+            return t.pin_memory().numpy()
+        except Exception:
+            return arr
+
+    class H:  # host CSR over pinned arrays
+        pass
+
+    def host_csr(M):
+        h = H()
+        h.n_rows, h.n_cols = M.n_rows, M.n_cols
+        h.row_ptr, h.col, h.val = pinned(M.row_ptr), pinned(M.col), pinned(M.val)
+        return h
+
+    hA = host_csr(A)
+    hB = hA if B is A else host_csr(B)
+    pin = True
+    try:
+        out_rp = torch.empty(A.n_rows + 1, dtype=torch.int64, pin_memory=True).numpy()
+        out_col = torch.empty(nnz, dtype=torch.int32, pin_memory=True).numpy()
+        out_val = torch.empty(nnz, dtype=torch.float32 if sv == 4 else torch.float64, pin_memory=True).numpy()
+    except Exception:
+        pin = False
+        out_rp = np.empty(A.n_rows + 1, np.int64)
+        out_col = np.empty(nnz, np.int32)
+        out_val = np.empty(nnz, A.val.dtype)
+    h2d = 2 * ((A.n_rows + 1) * 8 + A.nnz * (4 + sv)) if B is A else \
+        (A.n_rows + 1) * 8 + A.nnz * (4 + sv) + (B.n_rows + 1) * 8 + B.nnz * (4 + sv)
+    d2h = (A.n_rows + 1) * 8 + nnz * (4 + sv)
+    gm.spgemm_host(hA, hB, out_rp, out_col, out_val, SMEM_BYTES)  # warm-up
+    torch.cuda.synchronize()
+    t = time.perf_counter()
+    for _ in range(steps):
+        got = gm.spgemm_host(hA, hB, out_rp, out_col, out_val, SMEM_BYTES)
+    torch.cuda.synchronize()
+    dt = (time.perf_counter() - t) / steps
+    assert got == nnz and int(out_rp[-1]) == nnz
+    return {"value": 2.0 * products / dt / 1e9, "unit": "GFLOP/s", "h2d_bytes_per_step": int(h2d),
+            "d2h_bytes_per_step": int(d2h), "ms_per_step": dt * 1e3, "steps": steps, "pinned_host_buffers": pin,
+            "api": "gm_spgemm_host"}
+
+
+if __name__ == "__main__":
+    main()

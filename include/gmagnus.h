@@ -104,6 +104,7 @@ typedef struct gm_plan_info {
   int64_t stage_elems;     /* capacity of one staging half-buffer, in products                 */
   int64_t workspace_bytes; /* device memory held by the plan                                   */
   int64_t light_bin_rows[8]; /* light rows per size class of the symbolic pass                 */
+  int64_t launches;        /* kernels launched while planning                                  */
 } gm_plan_info;
 
 /* Filled by the most recent gm_spgemm_execute on the plan.  Times are CUDA-event milliseconds on
@@ -111,13 +112,14 @@ typedef struct gm_plan_info {
  * environment or through gm_plan_set_timing(plan, 1); otherwise they are 0. */
 typedef struct gm_exec_stats {
   int64_t c_nnz;
+  int64_t c_nnz_heavy;         /* entries of C that belong to heavy rows                       */
   int64_t c_capacity;          /* entries the C arrays have room for                           */
   int64_t staged_products;     /* products written to the staging buffer (all batches)         */
   int64_t final_chunks;        /* (row, chunk) pairs handed to the accumulate kernel           */
   int64_t launches;            /* kernels launched by this execute                             */
   float ms_light_symbolic, ms_light_numeric, ms_expand, ms_histogram, ms_multisplit,
       ms_acc_symbolic, ms_acc_numeric, ms_scan, ms_total;
-  float reserved[7];
+  float reserved[5];
 } gm_exec_stats;
 
 typedef struct gm_plan gm_plan; /* opaque, owned by the library */
@@ -136,6 +138,16 @@ int gm_set_allocator(gm_alloc_fn alloc_fn, gm_free_fn free_fn, void* user);
  * c_cols = C.m, opts may be NULL.  Errors: GM_ERR_INVALID_ARG, GM_ERR_UNSUPPORTED_SMEM. */
 int gm_planner_params(int64_t c_cols, int32_t dtype, size_t smem_bytes, const gm_plan_opts* opts,
                       gm_params* out);
+
+/* Host-only, no CUDA call: cuts the heavy rows into consecutive batches whose intermediate products
+ * fit one staging half-buffer (the paper keeps the whole intermediate matrix resident, Section
+ * III-A; batching is this library's addition for matrices whose intermediate matrix exceeds HBM).
+ * heavy_prefix: n_heavy + 1 exclusive prefix sums of IP_i over the heavy rows (host).  Writes the
+ * batch boundaries (heavy-row positions, first = 0, last = n_heavy) to bounds_out (room for
+ * max_bounds entries) and returns the number of batches, or GM_ERR_CAPACITY if one row alone
+ * exceeds stage_elems or bounds_out is too small.  A row is never split across batches. */
+int64_t gm_planner_batches(const int64_t* heavy_prefix, int64_t n_heavy, int64_t stage_elems,
+                           int64_t* bounds_out, int64_t max_bounds);
 
 /* Setup phase of Algorithm 3 (GetMagnusParams, InterOffsets, ThreshPartition) plus everything
  * else that depends only on the structure of A and B: counts the intermediate products of every

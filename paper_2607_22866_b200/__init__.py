@@ -9,6 +9,7 @@ from .binding import (  # noqa: F401
     Plan,
     DeviceCSR,
     planner_params,
+    planner_batches,
     spgemm_plan,
     spgemm_execute,
     spgemm,

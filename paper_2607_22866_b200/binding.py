@@ -19,7 +19,7 @@ from . import build as _build
 
 GM_MAX_LEVELS = 8
 EXPORTED_SYMBOLS = [
-    "gm_set_allocator", "gm_planner_params", "gm_spgemm_plan", "gm_spgemm_plan_ex", "gm_spgemm_execute",
+    "gm_set_allocator", "gm_planner_params", "gm_planner_batches", "gm_spgemm_plan", "gm_spgemm_plan_ex", "gm_spgemm_execute",
     "gm_spgemm_host", "gm_plan_get_info", "gm_exec_get_stats", "gm_plan_set_timing",
     "gm_plan_get_row_products", "gm_csr_free", "gm_plan_destroy", "gm_status_string", "gm_last_error",
 ]
@@ -62,16 +62,17 @@ class PlanInfo(ctypes.Structure):
                 ("products_max_row", ctypes.c_int64), ("rows_heavy", ctypes.c_int64),
                 ("rows_light", ctypes.c_int64), ("rows_empty", ctypes.c_int64), ("nnz_a_heavy", ctypes.c_int64),
                 ("c_nnz_upper", ctypes.c_int64), ("n_batches", ctypes.c_int64), ("stage_elems", ctypes.c_int64),
-                ("workspace_bytes", ctypes.c_int64), ("light_bin_rows", ctypes.c_int64 * 8)]
+                ("workspace_bytes", ctypes.c_int64), ("light_bin_rows", ctypes.c_int64 * 8),
+                ("launches", ctypes.c_int64)]
 
 
 class ExecStats(ctypes.Structure):
-    _fields_ = [("c_nnz", ctypes.c_int64), ("c_capacity", ctypes.c_int64), ("staged_products", ctypes.c_int64),
+    _fields_ = [("c_nnz", ctypes.c_int64), ("c_nnz_heavy", ctypes.c_int64), ("c_capacity", ctypes.c_int64), ("staged_products", ctypes.c_int64),
                 ("final_chunks", ctypes.c_int64), ("launches", ctypes.c_int64),
                 ("ms_light_symbolic", ctypes.c_float), ("ms_light_numeric", ctypes.c_float),
                 ("ms_expand", ctypes.c_float), ("ms_histogram", ctypes.c_float), ("ms_multisplit", ctypes.c_float),
                 ("ms_acc_symbolic", ctypes.c_float), ("ms_acc_numeric", ctypes.c_float), ("ms_scan", ctypes.c_float),
-                ("ms_total", ctypes.c_float), ("reserved", ctypes.c_float * 7)]
+                ("ms_total", ctypes.c_float), ("reserved", ctypes.c_float * 5)]
 
 
 _ALLOC_FN = ctypes.CFUNCTYPE(ctypes.c_void_p, ctypes.c_size_t, ctypes.c_void_p, ctypes.c_void_p)
@@ -109,6 +110,8 @@ def load_library(install_torch_allocator: bool = True):
         P = ctypes.POINTER
         lib.gm_set_allocator.argtypes = [_ALLOC_FN, _FREE_FN, vp]
         lib.gm_planner_params.argtypes = [i64, i32, sz, P(PlanOpts), P(Params)]
+        lib.gm_planner_batches.argtypes = [vp, i64, i64, vp, i64]
+        lib.gm_planner_batches.restype = i64
         lib.gm_spgemm_plan.argtypes = [P(_CSR), P(_CSR), sz, P(vp)]
         lib.gm_spgemm_plan_ex.argtypes = [P(_CSR), P(_CSR), sz, P(PlanOpts), vp, P(vp)]
         lib.gm_spgemm_execute.argtypes = [vp, vp, P(_CSR)]
@@ -176,6 +179,17 @@ def planner_params(c_cols: int, dtype, smem_bytes: int, opts: PlanOpts | None = 
     _check(load_library().gm_planner_params(c_cols, code, smem_bytes, ctypes.byref(opts) if opts else None,
                                             ctypes.byref(out)), "gm_planner_params")
     return out
+
+
+def planner_batches(heavy_prefix: np.ndarray, stage_elems: int) -> list[int]:
+    """gm_planner_batches: boundaries (heavy-row positions) of the staging-buffer batches."""
+    hp = np.ascontiguousarray(heavy_prefix, dtype=np.int64)
+    n = hp.size - 1
+    out = np.zeros(n + 2, dtype=np.int64)
+    rc = load_library().gm_planner_batches(hp.ctypes.data, n, stage_elems, out.ctypes.data, out.size)
+    if rc < 0:
+        raise GmError(int(rc), "gm_planner_batches", "a row exceeds stage_elems")
+    return out[: rc + 1].tolist()
 
 
 def _stream_ptr(stream) -> int:

@@ -239,6 +239,7 @@ static int build_plan(gm_plan* p, cudaStream_t st) {
       k_validate_csr<<<grid_for(M->n_rows, 256, p->num_sms), 256, 0, st>>>(M->row_ptr, M->col_idx, M->n_rows,
                                                                           M->n_cols, M->nnz, p->err + 1);
     }
+    info.launches += 2;
     int bad = 0;
     GM_CUDA(cudaMemcpyAsync(&bad, p->err + 1, sizeof(int), cudaMemcpyDeviceToHost, st));
     GM_CUDA(cudaStreamSynchronize(st));
@@ -266,6 +267,7 @@ static int build_plan(gm_plan* p, cudaStream_t st) {
                                                                   p->heavy_flag, totals);
   }
   exclusive_scan<int32_t, i64>(p->heavy_flag, heavy_pos, nA, p->scan_tmp, nullptr, nullptr, nullptr, st);
+  info.launches += (nnzA > 0 ? 3 : 1) + (nA > 0 ? 3 : 1) + (nA > 0 ? 2 : 0) + 1;
 
   // ---- light rows: bins by IP_i for the symbolic pass
   {
@@ -325,6 +327,7 @@ static int build_plan(gm_plan* p, cudaStream_t st) {
     k1_heavy_segments<<<grid_for(p->n_seg + 1, 256, p->num_sms, 32), 256, 0, st>>>(
         p->x_heavy, nH, p->heavy_nz_off, p->heavy_base, A.row_ptr, A.col_idx, p->nz_off, B.row_ptr, p->n_seg, p->seg_off,
         p->seg_bstart, p->seg_j);
+    info.launches += 8;
     std::vector<int64_t> hb(static_cast<size_t>(nH) + 1);
     p->x_heavy_host.resize(static_cast<size_t>(nH));
     GM_CUDA(cudaMemcpyAsync(hb.data(), p->heavy_base, hb.size() * sizeof(int64_t), cudaMemcpyDeviceToHost, st));
@@ -417,7 +420,10 @@ static int launch_light(gm_plan* p, const int32_t* rows_all, const int* fill_dev
 }
 
 __global__ void k_heavy_row_counts(const i64* __restrict__ chunk_nnz_off, int log2_chunks_per_row, i64 n_rows_b,
-                                   const int32_t* __restrict__ x_heavy, i64 h0, int32_t* __restrict__ row_nnz) {
+                                   const int32_t* __restrict__ x_heavy, i64 h0, int32_t* __restrict__ row_nnz,
+                                   i64* __restrict__ heavy_total) {
+  if (blockIdx.x == 0 && threadIdx.x == 0)
+    atomicAdd(reinterpret_cast<u64*>(heavy_total), static_cast<u64>(chunk_nnz_off[n_rows_b << log2_chunks_per_row]));
   for (i64 r = static_cast<i64>(blockIdx.x) * blockDim.x + threadIdx.x; r < n_rows_b;
        r += static_cast<i64>(gridDim.x) * blockDim.x) {
     row_nnz[x_heavy[h0 + r]] =
@@ -539,7 +545,7 @@ static int heavy_batch_front(gm_plan* p, const Batch& b, HeavyBatchState<V>* hs,
   tm.begin(PhaseTimes::kScan, st);
   exclusive_scan<u32, i64>(p->chunk_nnz, p->chunk_nnz_off, hs->n_chunks, p->scan_tmp, nullptr, nullptr, nullptr, st);
   k_heavy_row_counts<<<grid_for(rows_b, 256, p->num_sms), 256, 0, st>>>(p->chunk_nnz_off, hs->log2_cpr, rows_b, p->x_heavy,
-                                                                        b.h0, p->row_nnz);
+                                                                        b.h0, p->row_nnz, p->c_total + 1);
   p->stats.launches += 4;
   tm.end(st);
   return GM_OK;
@@ -610,6 +616,7 @@ static int execute_t(gm_plan* p, cudaStream_t st, gm_csr* C) {
   const size_t n_batches = p->batches.size();
   i64 capacity = 0;
   i64 total = 0;
+  i64 heavy_total = 0;
   int dev_err = 0;
   if (n_batches <= 1) {
     // ---- everything is resident at once: count, allocate C exactly, then fill
@@ -636,16 +643,33 @@ static int execute_t(gm_plan* p, cudaStream_t st, gm_csr* C) {
     GM_TRY_C(light_numeric(capacity));
   } else {
     // ---- heavy rows in several staging-buffer fills: C is appended in row order into reserved room
-    capacity = p->opts.c_capacity;
-    if (capacity <= 0) {
+    // Room for C.  Given: use it.  Derived: the structural upper bound sum_i min(IP_i, C.m), cut
+    // down to what the device can hold; if the allocator refuses (its own cache can hide free
+    // memory from cudaMemGetInfo, or the estimate was too bold) retry with less.
+    std::vector<i64> tries;
+    if (p->opts.c_capacity > 0) {
+      tries.push_back(p->opts.c_capacity);
+    } else {
       size_t free_b = 0, total_b = 0;
       GM_CUDA(cudaMemGetInfo(&free_b, &total_b));
-      const i64 reserve = i64{1} << 30;
-      const i64 by_mem = (static_cast<i64>(free_b) - reserve - (nA + 1) * 8) / static_cast<i64>(4 + sizeof(V));
-      capacity = std::min<i64>(info.c_nnz_upper, std::max<i64>(by_mem, 1));
+      const i64 entry = static_cast<i64>(4 + sizeof(V));
+      const i64 inputs = (A.nnz + (&A == &B ? 0 : B.nnz)) * entry + (A.n_rows + B.n_rows + 2) * 8;
+      const i64 by_total = (static_cast<i64>(total_b) - info.workspace_bytes - inputs - (nA + 1) * 8 - (i64{3} << 30)) / entry;
+      const i64 by_free = (static_cast<i64>(free_b) - (nA + 1) * 8 - (i64{1} << 30)) / entry;
+      const i64 hi = std::max<i64>(1, std::min<i64>(info.c_nnz_upper, std::max(by_total, by_free)));
+      const i64 lo = std::max<i64>(1, std::min<i64>(info.c_nnz_upper, by_free));
+      tries.push_back(hi);
+      for (int k = 1; k <= 3 && hi > lo; ++k) tries.push_back(hi - (hi - lo) * k / 3);
     }
-    c_col = static_cast<int32_t*>(dev_alloc(static_cast<size_t>(std::max<i64>(capacity, 1)) * sizeof(int32_t), st));
-    c_val = static_cast<V*>(dev_alloc(static_cast<size_t>(std::max<i64>(capacity, 1)) * sizeof(V), st));
+    for (i64 cand : tries) {
+      capacity = cand;
+      c_col = static_cast<int32_t*>(dev_alloc(static_cast<size_t>(capacity) * sizeof(int32_t), st));
+      c_val = c_col ? static_cast<V*>(dev_alloc(static_cast<size_t>(capacity) * sizeof(V), st)) : nullptr;
+      if (c_col && c_val) break;
+      dev_free(c_col, st);
+      c_col = nullptr;
+      c_val = nullptr;
+    }
     if (!c_col || !c_val) { cleanup(); return fail(GM_ERR_OOM, "allocation of C (room for " + std::to_string(capacity) + " entries) failed"); }
     for (size_t bi = 0; bi < n_batches; ++bi) {
       const Batch& b = p->batches[bi];
@@ -669,6 +693,7 @@ static int execute_t(gm_plan* p, cudaStream_t st, gm_csr* C) {
     }
   }
   if (tm.enabled) cudaEventRecord(ev_total1, st);
+  cudaMemcpyAsync(&heavy_total, p->c_total + 1, sizeof(i64), cudaMemcpyDeviceToHost, st);
   cudaError_t e1 = cudaMemcpyAsync(&dev_err, p->err, sizeof(int), cudaMemcpyDeviceToHost, st);
   cudaError_t e2 = cudaStreamSynchronize(st);
   if (e1 != cudaSuccess || e2 != cudaSuccess) {
@@ -682,6 +707,7 @@ static int execute_t(gm_plan* p, cudaStream_t st, gm_csr* C) {
   }
 #undef GM_TRY_C
   p->stats.c_nnz = total;
+  p->stats.c_nnz_heavy = heavy_total;
   p->stats.c_capacity = capacity;
   if (tm.enabled) {
     float ph[PhaseTimes::kCount];

@@ -64,13 +64,14 @@ __global__ void __launch_bounds__(BT) k6_accumulate(
       if (wb + i < n_words) local += __popc(bitmap[wb + i]);
     u32 total;
     u32 ex = block_exclusive_scan(local, s_scan, &total);
-    if (!NUMERIC) {
+    if constexpr (!NUMERIC) {
       for (int i = 0; i < words_per_thread; ++i)
         if (wb + i < n_words) bitmap[wb + i] = 0u;
       if (tid == 0) chunk_nnz[k] = total;
       __syncthreads();
       continue;
     }
+    if constexpr (NUMERIC) {
     for (int i = 0; i < words_per_thread; ++i) {
       if (wb + i < n_words) {
         word_prefix[wb + i] = ex;
@@ -100,6 +101,7 @@ __global__ void __launch_bounds__(BT) k6_accumulate(
       if (lane == 0) bitmap[w] = 0u;
     }
     __syncthreads();
+    }
   }
 }
 

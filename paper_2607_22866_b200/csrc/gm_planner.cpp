@@ -138,3 +138,14 @@ extern "C" int gm_planner_params(int64_t c_cols, int32_t dtype, size_t smem_byte
                                  const gm_plan_opts* opts, gm_params* out) {
   return gm::planner_params(c_cols, dtype, smem_bytes, opts, out);
 }
+
+extern "C" int64_t gm_planner_batches(const int64_t* heavy_prefix, int64_t n_heavy, int64_t stage_elems,
+                                      int64_t* bounds_out, int64_t max_bounds) {
+  if (!heavy_prefix || !bounds_out || n_heavy < 0 || stage_elems <= 0) return GM_ERR_INVALID_ARG;
+  std::vector<gm::Batch> b;
+  if (!gm::cut_batches(heavy_prefix, n_heavy, stage_elems, &b)) return GM_ERR_CAPACITY;
+  if (static_cast<int64_t>(b.size()) + 1 > max_bounds) return GM_ERR_CAPACITY;
+  bounds_out[0] = 0;
+  for (size_t i = 0; i < b.size(); ++i) bounds_out[i + 1] = b[i].h1;
+  return static_cast<int64_t>(b.size());
+}
