@@ -20,6 +20,8 @@
 
 namespace gm {
 
+static_assert(kAccTile == kAccTileElems && kAccMetaCap == kAccMetaEntries, "planner and kernel disagree");
+
 // ------------------------------------------------------------------------------------------------
 // errors, allocator
 // ------------------------------------------------------------------------------------------------
@@ -162,6 +164,9 @@ struct gm_plan {
   int64_t* level_off[2]{};         // max_batch_rows * chunks_required + 1 each (ping-pong)
   gm::u32* chunk_nnz = nullptr;
   int64_t* chunk_nnz_off = nullptr;
+  int64_t* chunk_base = nullptr;   // numeric pass: position in C of every chunk's first entry
+  int64_t* seg_first = nullptr;    // accumulate kernel: first chunk of every element segment
+  int* ticket = nullptr;
   gm::PhaseTimes times;
 };
 
@@ -351,7 +356,8 @@ static int build_plan(gm_plan* p, cudaStream_t st) {
       info.stage_elems = std::max(info.stage_elems, b.elems);
       p->max_batch_rows = std::max(p->max_batch_rows, b.h1 - b.h0);
     }
-    const size_t se = static_cast<size_t>(info.stage_elems);
+    // the accumulate kernel streams whole tiles: it may read (and ignore) up to one tile past the last product
+    const size_t se = static_cast<size_t>(info.stage_elems) + kAccTile + 8;
     const int n_buf = prm.n_levels > 0 ? 2 : 1;
     for (int i = 0; i < n_buf; ++i) {
       GM_TRY(plan_alloc(p, &p->stage_col[i], se, st));
@@ -368,6 +374,9 @@ static int build_plan(gm_plan* p, cudaStream_t st) {
     }
     GM_TRY(plan_alloc(p, &p->chunk_nnz, n_chunks_max + 1, st));
     GM_TRY(plan_alloc(p, &p->chunk_nnz_off, n_chunks_max + 1, st));
+    GM_TRY(plan_alloc(p, &p->chunk_base, n_chunks_max + 1, st));
+    GM_TRY(plan_alloc(p, &p->seg_first, static_cast<size_t>(info.stage_elems / kAccSegment) + 4, st));
+    GM_TRY(plan_alloc(p, &p->ticket, 4, st));
     int64_t* tmp2 = nullptr;  // the per-batch scans can be longer than the ones above
     GM_TRY(plan_alloc(p, &tmp2, static_cast<size_t>(scan_tmp_elems(std::max<i64>({static_cast<i64>(n_chunks_max), nnzA, nA, 1}))), st));
     p->scan_tmp = tmp2;
@@ -451,24 +460,36 @@ static int launch_accumulate(gm_plan* p, const Batch& b, const HeavyBatchState<V
                              int32_t* c_col, V* c_val, i64 c_capacity, cudaStream_t st) {
   const gm_params& prm = p->info.params;
   const int W = prm.chunk_width;
-  const size_t smem = acc_smem_bytes(W, sizeof(V), NUMERIC);
-  const int ctas = NUMERIC ? prm.acc_ctas_per_sm : 8;
-  const unsigned grid = static_cast<unsigned>(std::min<i64>(hs.n_chunks, static_cast<i64>(p->num_sms) * ctas));
+  const int ctas = prm.acc_ctas_per_sm;
+  const size_t budget = p->smem_bytes / static_cast<size_t>(ctas) - 1024;
+  const int stages = acc_ring_stages(budget, W, sizeof(V), NUMERIC);
+  if (stages < 2) return fail(GM_ERR_UNSUPPORTED_SMEM, "shared memory budget too small for the accumulate kernel");
+  const size_t smem = acc_stream_smem_bytes(W, sizeof(V), NUMERIC, stages);
+  const i64 n_segs = (b.elems + kAccSegment - 1) / kAccSegment;
+  const i64 prep = std::max<i64>(n_segs + 1, NUMERIC ? hs.n_chunks : 0);
+  k6_prepare<<<static_cast<unsigned>((prep + 255) / 256), 256, 0, st>>>(
+      hs.chunk_off, hs.n_chunks, n_segs, p->seg_first, p->chunk_nnz_off, hs.log2_cpr, p->x_heavy, b.h0, c_row_ptr,
+      NUMERIC ? p->chunk_base : nullptr);
+  GM_CUDA(cudaMemsetAsync(p->ticket, 0, sizeof(int), st));
+  if (!NUMERIC) GM_CUDA(cudaMemsetAsync(p->chunk_nnz, 0, static_cast<size_t>(hs.n_chunks) * sizeof(u32), st));
+  // symbolic launches keep only a bitmap next to the ring, so two blocks share an SM
+  const int per_sm = NUMERIC ? ctas : std::max(2, ctas);
+  const unsigned grid = static_cast<unsigned>(std::min<i64>(n_segs, static_cast<i64>(p->num_sms) * per_sm));
 #define GM_ACC(BT)                                                                                                    \
   do {                                                                                                                \
     auto kern = k6_accumulate<V, NUMERIC, BT>;                                                                        \
     if (smem > 48 * 1024)                                                                                             \
       GM_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)));      \
-    kern<<<grid, BT, smem, st>>>(hs.fin_col, hs.fin_val, hs.chunk_off, hs.n_chunks, hs.log2_cpr, W, p->B.n_cols,      \
-                                 p->chunk_nnz, p->chunk_nnz_off, p->x_heavy, b.h0, c_row_ptr, c_col, c_val, c_capacity, \
+    kern<<<grid, BT, smem, st>>>(hs.fin_col, hs.fin_val, hs.chunk_off, hs.n_chunks, p->seg_first, n_segs, p->ticket, \
+                                 hs.log2_cpr, W, stages, p->chunk_nnz, p->chunk_base, c_col, c_val, c_capacity,       \
                                  p->err);                                                                             \
   } while (0)
-  if (!NUMERIC) GM_ACC(256);
-  else if (prm.acc_ctas_per_sm == 1) GM_ACC(1024);
-  else if (prm.acc_ctas_per_sm == 2) GM_ACC(512);
+  // 1024 threads per SM in total: the floating-point shared-memory atomics are latency bound
+  if (ctas == 1) GM_ACC(1024);
+  else if (ctas == 2) GM_ACC(512);
   else GM_ACC(256);
 #undef GM_ACC
-  ++p->stats.launches;
+  p->stats.launches += 2;
   GM_CUDA(cudaGetLastError());
   return GM_OK;
 }
@@ -557,6 +578,7 @@ static int dev_error_to_status(int code) {
     case kDevCapacity: return fail(GM_ERR_CAPACITY, "C did not fit the room reserved for it (raise c_capacity or stage fewer products)");
     case kDevTableFull: return fail(GM_ERR_INTERNAL, "a light-row hash table overflowed");
     case kDevBadChunk: return fail(GM_ERR_INTERNAL, "an intermediate product reached a chunk that does not own its column");
+    case kDevTimeout: return fail(GM_ERR_TIMEOUT, "a bounded wait on an asynchronous copy gave up");
     default: return fail(GM_ERR_INTERNAL, "unknown device error code");
   }
 }

@@ -16,6 +16,7 @@ enum DevError : int {
   kDevCapacity = 1,      // a write would have gone past the room reserved for C
   kDevTableFull = 2,     // a light-row hash table overflowed (planner bug)
   kDevBadChunk = 3,      // an element landed in a chunk that does not own its column
+  kDevTimeout = 4,       // a bounded wait on an asynchronous copy gave up
 };
 
 __device__ __forceinline__ void dev_set_error(int* flag, int code) { atomicCAS(flag, 0, code); }

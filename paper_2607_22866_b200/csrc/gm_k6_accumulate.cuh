@@ -6,101 +6,319 @@
 // ascending column order at   C.rowPtr[row] + (entries of the row's earlier chunks) + rank.
 //   symbolic launch: bitmap only -> entries per chunk (feeds C.rowPtr)
 //   numeric launch : values + bitmap -> C.col / C.val
-// Blocks are persistent and take chunks in a strided order; the accumulator is cleaned while it is
-// written out, so a chunk costs time proportional to its products and its output, not to W.
+//
+// B200 design.  The chunks of a batch lie back to back in the staging buffer, so the kernel does
+// not fetch chunk by chunk: the element space is cut into equal segments (static flattened
+// partition, as in Algorithms 4 and 5), persistent blocks claim segments with a ticket, and each
+// block *streams* its segment through a ring of shared-memory tiles filled by bulk asynchronous
+// copies (cp.async.bulk + mbarrier), independent of chunk boundaries.  A chunk boundary only
+// triggers a flush of the accumulator.  The flush cleans what it writes, so a chunk costs time
+// proportional to its products and its output, not to W.  All waits are bounded.
 #pragma once
 #include "gm_common.cuh"
 
 namespace gm {
 
+constexpr int kAccTile = 2048;          // elements per ring stage
+constexpr int kAccMetaCap = 1024;       // chunk offsets / bases staged per refill
+constexpr i64 kAccSegment = i64{1} << 18;  // elements per ticket
+constexpr int kAccSpinLimit = 1 << 24;  // polls of an mbarrier before the kernel gives up
+
+__device__ __forceinline__ u32 smem_u32(const void* p) { return static_cast<u32>(__cvta_generic_to_shared(p)); }
+
+__device__ __forceinline__ void mbar_init(u64* bar, int count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(u64* bar, u32 bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(u64* bar, u32 parity) {
+  u32 ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(smem_u32(bar)), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+// 1-D bulk copy global -> this block's shared memory; both addresses 16-byte aligned, bytes a multiple of 16
+__device__ __forceinline__ void bulk_g2s(void* dst, const void* src, u32 bytes, u64* bar) {
+  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(smem_u32(dst)),
+               "l"(src), "r"(bytes), "r"(smem_u32(bar))
+               : "memory");
+}
+
+// Number of ring stages that fit next to the accumulator.
+__host__ __device__ inline int acc_ring_stages(size_t smem_budget, int W, int val_bytes, bool numeric) {
+  const size_t fixed = static_cast<size_t>(W / 32) * 8 + (numeric ? static_cast<size_t>(W) * val_bytes : 0) +
+                       static_cast<size_t>(kAccMetaCap) * (4 + (numeric ? 8 : 0)) + 256;
+  const size_t stage = static_cast<size_t>(kAccTile) * (4 + (numeric ? val_bytes : 0));
+  if (smem_budget <= fixed) return 0;
+  size_t s = (smem_budget - fixed) / stage;
+  return static_cast<int>(s > 8 ? 8 : s);
+}
+__host__ __device__ inline size_t acc_stream_smem_bytes(int W, int val_bytes, bool numeric, int stages) {
+  return static_cast<size_t>(W / 32) * 8 + (numeric ? static_cast<size_t>(W) * val_bytes : 0) +
+         static_cast<size_t>(kAccMetaCap) * (4 + (numeric ? 8 : 0)) +
+         static_cast<size_t>(stages) * kAccTile * (4 + (numeric ? val_bytes : 0)) + 256;
+}
+
+// seg_first[s] = first chunk whose start offset is >= s * kAccSegment (s = 0..n_segs); for the numeric
+// pass also the position in C of every chunk's first entry.
+__global__ void k6_prepare(const i64* __restrict__ chunk_off, i64 n_chunks, i64 n_segs, i64* __restrict__ seg_first,
+                           const i64* __restrict__ chunk_nnz_off, int log2_chunks_per_row,
+                           const int32_t* __restrict__ x_heavy, i64 h0, const i64* __restrict__ c_row_ptr,
+                           i64* __restrict__ chunk_base) {
+  const i64 i = static_cast<i64>(blockIdx.x) * blockDim.x + threadIdx.x;
+  if (i <= n_segs) {
+    const i64 target = i * kAccSegment;
+    i64 lo = 0, hi = n_chunks;  // first k in [0, n_chunks] with chunk_off[k] >= target
+    while (lo < hi) {
+      const i64 mid = (lo + hi) >> 1;
+      if (chunk_off[mid] >= target) hi = mid; else lo = mid + 1;
+    }
+    seg_first[i] = lo;
+  }
+  if (chunk_base && i < n_chunks) {
+    const i64 r = i >> log2_chunks_per_row;
+    chunk_base[i] = c_row_ptr[x_heavy[h0 + r]] + (chunk_nnz_off[i] - chunk_nnz_off[r << log2_chunks_per_row]);
+  }
+}
+
+// One product into the accumulator.  Measured on B200 (shared memory, 1024 threads per SM, products per clock
+// per SM): native integer atomics 12; floating-point atomicAdd (a compare-and-swap loop) 3.7 on uniform
+// columns and 2.0 when a quarter of the products hit 64 hot columns; ranking equal columns first with a warp
+// match (match.any) only 0.5 — so there is no warp-level deduplication here, and the bitmap is tested before
+// it is set so that repeated columns cost a load instead of an atomic.
+template <typename V, bool NUMERIC>
+__device__ __forceinline__ void acc_add(bool valid, u32 cl, V v, V* acc, u32* bitmap) {
+  if (valid) {
+    if constexpr (NUMERIC) atomicAdd(&acc[cl], v);
+    const u32 bit = 1u << (cl & 31);
+    if (!(bitmap[cl >> 5] & bit)) atomicOr(&bitmap[cl >> 5], bit);
+  }
+}
+
 template <typename V, bool NUMERIC, int BT>
 __global__ void __launch_bounds__(BT) k6_accumulate(
     const int32_t* __restrict__ x_col, const V* __restrict__ x_val,
-    const i64* __restrict__ chunk_off,   // n_chunks + 1, batch-relative element offsets
-    i64 n_chunks, int log2_chunks_per_row, int W, i64 c_cols,
-    u32* __restrict__ chunk_nnz,                     // symbolic out
-    const i64* __restrict__ chunk_nnz_off,           // numeric in: exclusive scan of chunk_nnz (n_chunks + 1)
-    const int32_t* __restrict__ x_heavy, i64 h0,     // heavy rows of the batch: original row = x_heavy[h0 + r]
-    const i64* __restrict__ c_row_ptr, int32_t* __restrict__ c_col, V* __restrict__ c_val, i64 c_capacity,
-    int* __restrict__ err) {
-  extern __shared__ __align__(16) unsigned char smem_raw[];
+    const i64* __restrict__ chunk_off,   // n_chunks + 1 batch-relative element offsets
+    i64 n_chunks, const i64* __restrict__ seg_first, i64 n_segs, int* __restrict__ ticket,
+    int log2_chunks_per_row, int W, int stages,
+    u32* __restrict__ chunk_nnz,                 // symbolic out (pre-zeroed: empty chunks are never visited)
+    const i64* __restrict__ chunk_base,          // numeric in: position in C of the chunk's first entry
+    int32_t* __restrict__ c_col, V* __restrict__ c_val, i64 c_capacity, int* __restrict__ err) {
+  extern __shared__ __align__(128) unsigned char smem_acc_raw[];
   const int n_words = W >> 5;
-  V* acc = reinterpret_cast<V*>(smem_raw);
-  u32* bitmap = reinterpret_cast<u32*>(smem_raw + (NUMERIC ? static_cast<size_t>(W) * sizeof(V) : 0));
-  u32* word_prefix = bitmap + n_words;
+  // layout: [ring cols][ring vals][acc][bitmap][meta base (i64)][meta off (i32)]
+  int32_t* r_col = reinterpret_cast<int32_t*>(smem_acc_raw);
+  V* r_val = reinterpret_cast<V*>(smem_acc_raw + static_cast<size_t>(stages) * kAccTile * 4);
+  unsigned char* after_ring = smem_acc_raw + static_cast<size_t>(stages) * kAccTile * (4 + (NUMERIC ? sizeof(V) : 0));
+  V* acc = reinterpret_cast<V*>(after_ring);
+  u32* bitmap = reinterpret_cast<u32*>(after_ring + (NUMERIC ? static_cast<size_t>(W) * sizeof(V) : 0));
+  i64* m_base = reinterpret_cast<i64*>(bitmap + 2 * n_words);
+  int* m_off = reinterpret_cast<int*>(m_base + (NUMERIC ? kAccMetaCap : 0));
+  __shared__ u64 full_bar[8];
   __shared__ u32 s_scan[33];
-  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  constexpr int kWarps = BT / 32;
+  __shared__ i64 s_seg[2];
+  __shared__ int s_abort;
+
+  const int tid = threadIdx.x, lane = tid & 31;
   const u32 wmask = static_cast<u32>(W - 1);
+  constexpr u32 kStageBytesCol = kAccTile * 4;
+  constexpr u32 kStageBytesVal = NUMERIC ? kAccTile * sizeof(V) : 0;
+  constexpr int kPerThread = kAccTile / BT;  // elements of a full tile per thread
+  static_assert(kAccTile % BT == 0, "tile must be a multiple of the block");
+  // the flush gives every thread wpt consecutive bitmap words (wpt is a power of two, at most 32)
+  const int wpt = n_words > BT ? n_words / BT : 1;
 
   if (NUMERIC)
     for (int s = tid; s < W; s += BT) acc[s] = V(0);
   for (int w = tid; w < n_words; w += BT) bitmap[w] = 0u;
+  if (tid == 0) {
+    for (int s = 0; s < stages; ++s) mbar_init(&full_bar[s], 1);
+    s_abort = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
   __syncthreads();
+  u32 phase_bits = 0;  // bit s = parity to wait for on stage s
 
-  const int words_per_thread = (n_words + BT - 1) / BT;
-  for (i64 k = blockIdx.x; k < n_chunks; k += gridDim.x) {
-    const i64 e0 = chunk_off[k], e1 = chunk_off[k + 1];
-    if (e0 == e1) {
-      if (!NUMERIC && tid == 0) chunk_nnz[k] = 0u;
-      continue;
-    }
-    const i64 chunk = k & ((i64{1} << log2_chunks_per_row) - 1);
-    const i64 col_base = chunk * W;
-    // ---- accumulate
-    for (i64 e = e0 + tid; e < e1; e += BT) {
-      const u32 c = static_cast<u32>(x_col[e]);
-      const u32 cl = c & wmask;
-      if (static_cast<i64>(c) - cl != col_base) { dev_set_error(err, kDevBadChunk); continue; }
-      if (NUMERIC) atomicAdd(&acc[cl], x_val[e]);
-      const u32 bit = 1u << (cl & 31);
-      if (!(bitmap[cl >> 5] & bit)) atomicOr(&bitmap[cl >> 5], bit);
+  for (;;) {
+    if (tid == 0) {
+      const int s = atomicAdd(ticket, 1);
+      s_seg[0] = s < n_segs ? seg_first[s] : -1;
+      s_seg[1] = s < n_segs ? seg_first[s + 1] : -1;
     }
     __syncthreads();
-    // ---- rank the occupied columns: popcount per bitmap word, block-wide exclusive scan
-    u32 local = 0;
-    const int wb = tid * words_per_thread;
-    for (int i = 0; i < words_per_thread; ++i)
-      if (wb + i < n_words) local += __popc(bitmap[wb + i]);
-    u32 total;
-    u32 ex = block_exclusive_scan(local, s_scan, &total);
-    if constexpr (!NUMERIC) {
-      for (int i = 0; i < words_per_thread; ++i)
-        if (wb + i < n_words) bitmap[wb + i] = 0u;
-      if (tid == 0) chunk_nnz[k] = total;
-      __syncthreads();
-      continue;
-    }
-    if constexpr (NUMERIC) {
-    for (int i = 0; i < words_per_thread; ++i) {
-      if (wb + i < n_words) {
-        word_prefix[wb + i] = ex;
-        ex += __popc(bitmap[wb + i]);
+    const i64 k_first = s_seg[0], k_end = s_seg[1];
+    __syncthreads();
+    if (k_first < 0) break;
+    if (k_first >= k_end) continue;
+    const i64 lo = chunk_off[k_first], hi = chunk_off[k_end];
+    if (lo >= hi) continue;
+    const i64 lo_al = lo & ~i64{3};  // 16-byte aligned start of the stream
+    const int n_tiles = static_cast<int>((hi - lo_al + kAccTile - 1) / kAccTile);
+    const int32_t* g_col = x_col + lo_al;
+    const V* g_val = x_val + lo_al;
+
+    auto issue = [&](int j, int st) {  // thread 0 only
+      const size_t g = static_cast<size_t>(j) * kAccTile;
+      mbar_expect_tx(&full_bar[st], kStageBytesCol + kStageBytesVal);
+      bulk_g2s(r_col + st * kAccTile, g_col + g, kStageBytesCol, &full_bar[st]);
+      if (NUMERIC) bulk_g2s(r_val + st * kAccTile, g_val + g, kStageBytesVal, &full_bar[st]);
+    };
+    if (tid == 0)
+      for (int j = 0; j < n_tiles && j < stages; ++j) issue(j, j);
+
+    // chunk metadata of the segment, refilled every kAccMetaCap chunks
+    i64 m0 = k_first;          // first chunk held in the metadata window
+    int kw = 0;                // current chunk = m0 + kw
+    auto load_meta = [&]() {
+      for (int i = tid; i < kAccMetaCap; i += BT) {
+        const i64 kk = m0 + i;
+        if (kk <= k_end) m_off[i] = static_cast<int>(chunk_off[kk] - lo_al);
+        if (NUMERIC && kk < k_end) m_base[i] = chunk_base[kk];
       }
-    }
+    };
+    load_meta();
     __syncthreads();
-    // ---- write out in column order and clean the accumulator
-    const i64 row_in_batch = k >> log2_chunks_per_row;
-    const i64 row = x_heavy[h0 + row_in_batch];
-    const i64 out0 = c_row_ptr[row] + (chunk_nnz_off[k] - chunk_nnz_off[row_in_batch << log2_chunks_per_row]);
-    const bool fits = out0 + total <= c_capacity;
-    if (!fits) dev_set_error(err, kDevCapacity);
-    for (int w = warp; w < n_words; w += kWarps) {
-      const u32 word = bitmap[w];
-      if (word == 0u) continue;
-      if ((word >> lane) & 1u) {
-        const int slot = (w << 5) + lane;
-        if (fits) {
-          const i64 pos = out0 + word_prefix[w] + __popc(word & lanemask_lt());
-          c_col[pos] = static_cast<int32_t>(col_base + slot);
-          c_val[pos] = acc[slot];
+
+    int pos = static_cast<int>(lo - lo_al);      // stream-relative position of the next element
+    const int end = static_cast<int>(hi - lo_al);
+    bool aborted = false;
+    int st = 0;
+
+    for (int j = 0; j < n_tiles; ++j) {
+      // ---- wait for the tile (bounded, with back-off so that the poll does not eat issue slots)
+      {
+        const u32 par = (phase_bits >> st) & 1u;
+        int spins = 0;
+        while (!mbar_try_wait(&full_bar[st], par)) {
+          __nanosleep(40);
+          if (++spins > kAccSpinLimit) { s_abort = 1; break; }
         }
-        acc[slot] = V(0);
+        phase_bits ^= (1u << st);
       }
-      __syncwarp();
-      if (lane == 0) bitmap[w] = 0u;
+      const int tile_lo = j * kAccTile;
+      const int tile_hi = min(end, tile_lo + kAccTile);
+      const int32_t* tc = r_col + st * kAccTile - tile_lo;
+      const V* tv = r_val + st * kAccTile - tile_lo;
+      while (pos < tile_hi) {
+        // make sure the current chunk and its end are inside the metadata window
+        if (kw + 1 >= kAccMetaCap) {
+          __syncthreads();
+          m0 += kw;
+          kw = 0;
+          load_meta();
+          __syncthreads();
+        }
+        const int ce = m_off[kw + 1];
+        if (ce <= pos) { ++kw; continue; }  // empty chunk
+        const int sub_hi = min(tile_hi, ce);
+        const u32 col_base = static_cast<u32>((m0 + kw) & ((i64{1} << log2_chunks_per_row) - 1)) * static_cast<u32>(W);
+        if (!s_abort) {
+          for (int base = pos; base < sub_hi; base += BT * kPerThread) {
+            u32 cl[kPerThread];
+            V v[kPerThread];
+            bool ok[kPerThread];
+#pragma unroll
+            for (int u = 0; u < kPerThread; ++u) {
+              const int q = base + u * BT + tid;
+              ok[u] = q < sub_hi;
+              u32 c = col_base;
+              v[u] = V(0);
+              if (ok[u]) {
+                c = static_cast<u32>(tc[q]);
+                if (NUMERIC) v[u] = tv[q];
+              }
+              cl[u] = c & wmask;
+              if (c - cl[u] != col_base) { dev_set_error(err, kDevBadChunk); ok[u] = false; }
+            }
+#pragma unroll
+            for (int u = 0; u < kPerThread; ++u) acc_add<V, NUMERIC>(ok[u], cl[u], v[u], acc, bitmap);
+          }
+        }
+        pos = sub_hi;
+        if (pos < ce) break;  // chunk continues in the next tile
+        // ---- chunk complete: flush
+        __syncthreads();
+        const int wb = tid * wpt;
+        u32 pc = 0;
+        if (wb < n_words)
+          for (int i = 0; i < wpt; ++i) pc += __popc(bitmap[wb + i]);
+        u32 total;
+        u32 ex = block_exclusive_scan(pc, s_scan, &total);
+        if constexpr (!NUMERIC) {
+          if (wb < n_words)
+            for (int i = 0; i < wpt; ++i) bitmap[wb + i] = 0u;
+          if (tid == 0) chunk_nnz[m0 + kw] = total;
+        } else {
+          const i64 out0 = m_base[kw];
+          const bool fits = out0 + total <= c_capacity;
+          if (!fits && tid == 0) dev_set_error(err, kDevCapacity);
+          for (int i = 0; i < wpt; ++i) {
+            // words with few bits: their owner writes them; dense words: the whole warp writes one word at a time
+            u32 word = 0;
+            if (wb < n_words) word = bitmap[wb + i];
+            const u32 wpc = __popc(word);
+            const bool dense = wpc > 4;
+            if (wpc && !dense) {
+              u32 wbits = word;
+              i64 p = out0 + ex;
+              while (wbits) {
+                const int b = __ffs(wbits) - 1;
+                wbits &= wbits - 1;
+                const int slot = ((wb + i) << 5) + b;
+                if (fits) { c_col[p] = static_cast<int32_t>(col_base + slot); c_val[p] = acc[slot]; }
+                acc[slot] = V(0);
+                ++p;
+              }
+            }
+            u32 dmask = __ballot_sync(0xffffffffu, dense);
+            while (dmask) {
+              const int src = __ffs(dmask) - 1;
+              dmask &= dmask - 1;
+              const u32 wd = __shfl_sync(0xffffffffu, word, src);
+              const u32 wex = __shfl_sync(0xffffffffu, ex, src);
+              const int wi = __shfl_sync(0xffffffffu, wb + i, src);
+              if ((wd >> lane) & 1u) {
+                const int slot = (wi << 5) + lane;
+                if (fits) {
+                  const i64 p = out0 + wex + __popc(wd & lanemask_lt());
+                  c_col[p] = static_cast<int32_t>(col_base + slot);
+                  c_val[p] = acc[slot];
+                }
+                acc[slot] = V(0);
+              }
+            }
+            if (wb < n_words) bitmap[wb + i] = 0u;
+            ex += wpc;
+          }
+        }
+        __syncthreads();
+        ++kw;
+      }
+      // ---- the stage is free again: refill it
+      __syncthreads();
+      if (s_abort) { aborted = true; break; }
+      if (tid == 0 && j + stages < n_tiles) issue(j + stages, st);
+      st = (st + 1 == stages) ? 0 : st + 1;
     }
-    __syncthreads();
+    if (aborted) {
+      // Tiles that were issued but not consumed still target this block's shared memory: give each a
+      // bounded chance to land before the block exits (its barrier answers at once if it already did).
+      if (tid == 0) {
+        dev_set_error(err, kDevTimeout);
+        for (int s2 = 0; s2 < stages; ++s2) {
+          int spins = 0;
+          while (!mbar_try_wait(&full_bar[s2], (phase_bits >> s2) & 1u) && ++spins < (1 << 20)) {
+          }
+        }
+      }
+      __syncthreads();
+      return;
     }
   }
 }

@@ -16,8 +16,11 @@ size_t light_smem_bytes(int64_t slots, int64_t cap, int val_bytes, bool numeric)
 }
 
 size_t acc_smem_bytes(int64_t W, int val_bytes, bool numeric) {
-  // bitmap (1 bit per column) + per-word prefix counts + (numeric: one value per column)
-  size_t b = static_cast<size_t>(W / 32) * 8 + 64;
+  // bitmap (1 bit per column) + per-word prefix counts + (numeric: one value per column), plus what the
+  // streaming needs at least: the chunk-metadata window and two ring stages of kAccTileElems products
+  size_t b = static_cast<size_t>(W / 32) * 8 + 256;
+  b += static_cast<size_t>(kAccMetaEntries) * (numeric ? 12 : 4);
+  b += 2 * static_cast<size_t>(kAccTileElems) * (numeric ? 4 + val_bytes : 4);
   if (numeric) b += static_cast<size_t>(W) * val_bytes;
   return b;
 }

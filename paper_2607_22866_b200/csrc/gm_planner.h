@@ -9,6 +9,8 @@ namespace gm {
 
 constexpr int kMultisplitBinCap = 2048;  // (parent, child) bins one multisplit tile keeps in smem
 constexpr int kMinSmemBytes = 16384;
+constexpr int kAccTileElems = 2048;    // products per ring stage of the accumulate kernel
+constexpr int kAccMetaEntries = 1024;  // chunk offsets / bases staged per refill
 
 inline int ilog2_floor(uint64_t x) {
   int l = 0;
