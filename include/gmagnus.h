@@ -68,7 +68,7 @@ typedef struct gm_plan_opts {
   int64_t tau;             /* heavy-row threshold: row i is heavy iff IP_i > tau               */
   int32_t chunk_width;     /* W: columns per final chunk (power of two)                        */
   int32_t max_fanout;      /* n_chunksMax: most children one multisplit level may produce (pow2) */
-  int32_t acc_ctas_per_sm; /* 1, 2 or 4: how many chunk accumulators share one SM (sets W)     */
+  int32_t acc_ctas_per_sm; /* 1, 2, 4 or 8: how many chunk accumulators share one SM (sets W)  */
   int64_t stage_elems;     /* capacity, in intermediate products, of each staging half-buffer  */
   int64_t c_capacity;      /* room, in entries, reserved for C when heavy rows need > 1 batch  */
   int32_t separate_histogram; /* 1: always run the stand-alone histogram kernel per level      */
@@ -88,7 +88,7 @@ typedef struct gm_params {
   int32_t fanout[GM_MAX_LEVELS]; /* v_chunks: children per parent at each level                */
   int32_t shift[GM_MAX_LEVELS];  /* child at level l = (col >> shift[l]) & (fanout[l] - 1)     */
   int32_t acc_ctas_per_sm;
-  int32_t reserved;
+  int32_t acc_block_threads; /* threads of one accumulate block                                  */
 } gm_params;
 
 typedef struct gm_plan_info {

@@ -50,7 +50,7 @@ class Params(ctypes.Structure):
     _fields_ = [("tau", ctypes.c_int64), ("light_slots", ctypes.c_int32), ("chunk_width", ctypes.c_int32),
                 ("chunks_required", ctypes.c_int32), ("max_fanout", ctypes.c_int32), ("n_levels", ctypes.c_int32),
                 ("fanout", ctypes.c_int32 * GM_MAX_LEVELS), ("shift", ctypes.c_int32 * GM_MAX_LEVELS),
-                ("acc_ctas_per_sm", ctypes.c_int32), ("reserved", ctypes.c_int32)]
+                ("acc_ctas_per_sm", ctypes.c_int32), ("acc_block_threads", ctypes.c_int32)]
 
     def levels(self):
         return [int(self.fanout[i]) for i in range(self.n_levels)]

@@ -20,8 +20,6 @@
 
 namespace gm {
 
-static_assert(kAccTile == kAccTileElems && kAccMetaCap == kAccMetaEntries, "planner and kernel disagree");
-
 // ------------------------------------------------------------------------------------------------
 // errors, allocator
 // ------------------------------------------------------------------------------------------------
@@ -167,6 +165,7 @@ struct gm_plan {
   int64_t* chunk_base = nullptr;   // numeric pass: position in C of every chunk's first entry
   int64_t* seg_first = nullptr;    // accumulate kernel: first chunk of every element segment
   int* ticket = nullptr;
+  gm::TileMeta* tile_meta = nullptr;  // per tile of the expansion / multisplit kernels: groups it touches
   gm::PhaseTimes times;
 };
 
@@ -357,7 +356,7 @@ static int build_plan(gm_plan* p, cudaStream_t st) {
       p->max_batch_rows = std::max(p->max_batch_rows, b.h1 - b.h0);
     }
     // the accumulate kernel streams whole tiles: it may read (and ignore) up to one tile past the last product
-    const size_t se = static_cast<size_t>(info.stage_elems) + kAccTile + 8;
+    const size_t se = static_cast<size_t>(info.stage_elems) + 2048 + 8;
     const int n_buf = prm.n_levels > 0 ? 2 : 1;
     for (int i = 0; i < n_buf; ++i) {
       GM_TRY(plan_alloc(p, &p->stage_col[i], se, st));
@@ -377,6 +376,8 @@ static int build_plan(gm_plan* p, cudaStream_t st) {
     GM_TRY(plan_alloc(p, &p->chunk_base, n_chunks_max + 1, st));
     GM_TRY(plan_alloc(p, &p->seg_first, static_cast<size_t>(info.stage_elems / kAccSegment) + 4, st));
     GM_TRY(plan_alloc(p, &p->ticket, 4, st));
+    const size_t n_tiles_max = static_cast<size_t>(info.stage_elems) / std::min(kExpandTile, kSplitTile) + 2;
+    GM_TRY(plan_alloc(p, &p->tile_meta, n_tiles_max, st));
     int64_t* tmp2 = nullptr;  // the per-batch scans can be longer than the ones above
     GM_TRY(plan_alloc(p, &tmp2, static_cast<size_t>(scan_tmp_elems(std::max<i64>({static_cast<i64>(n_chunks_max), nnzA, nA, 1}))), st));
     p->scan_tmp = tmp2;
@@ -462,9 +463,10 @@ static int launch_accumulate(gm_plan* p, const Batch& b, const HeavyBatchState<V
   const int W = prm.chunk_width;
   const int ctas = prm.acc_ctas_per_sm;
   const size_t budget = p->smem_bytes / static_cast<size_t>(ctas) - 1024;
-  const int stages = acc_ring_stages(budget, W, sizeof(V), NUMERIC);
+  const int bt = prm.acc_block_threads;
+  const int stages = acc_ring_stages(budget, W, sizeof(V), NUMERIC, bt);
   if (stages < 2) return fail(GM_ERR_UNSUPPORTED_SMEM, "shared memory budget too small for the accumulate kernel");
-  const size_t smem = acc_stream_smem_bytes(W, sizeof(V), NUMERIC, stages);
+  const size_t smem = acc_stream_smem_bytes(W, sizeof(V), NUMERIC, stages, bt);
   const i64 n_segs = (b.elems + kAccSegment - 1) / kAccSegment;
   const i64 prep = std::max<i64>(n_segs + 1, NUMERIC ? hs.n_chunks : 0);
   k6_prepare<<<static_cast<unsigned>((prep + 255) / 256), 256, 0, st>>>(
@@ -473,7 +475,7 @@ static int launch_accumulate(gm_plan* p, const Batch& b, const HeavyBatchState<V
   GM_CUDA(cudaMemsetAsync(p->ticket, 0, sizeof(int), st));
   if (!NUMERIC) GM_CUDA(cudaMemsetAsync(p->chunk_nnz, 0, static_cast<size_t>(hs.n_chunks) * sizeof(u32), st));
   // symbolic launches keep only a bitmap next to the ring, so two blocks share an SM
-  const int per_sm = NUMERIC ? ctas : std::max(2, ctas);
+  const int per_sm = (NUMERIC ? 1024 : 2048) / bt;  // a symbolic block needs no value array: twice as many fit
   const unsigned grid = static_cast<unsigned>(std::min<i64>(n_segs, static_cast<i64>(p->num_sms) * per_sm));
 #define GM_ACC(BT)                                                                                                    \
   do {                                                                                                                \
@@ -485,9 +487,10 @@ static int launch_accumulate(gm_plan* p, const Batch& b, const HeavyBatchState<V
                                  p->err);                                                                             \
   } while (0)
   // 1024 threads per SM in total: the floating-point shared-memory atomics are latency bound
-  if (ctas == 1) GM_ACC(1024);
-  else if (ctas == 2) GM_ACC(512);
-  else GM_ACC(256);
+  if (bt == 1024) GM_ACC(1024);
+  else if (bt == 512) GM_ACC(512);
+  else if (bt == 256) GM_ACC(256);
+  else GM_ACC(128);
 #undef GM_ACC
   p->stats.launches += 2;
   GM_CUDA(cudaGetLastError());
@@ -505,7 +508,10 @@ static int heavy_batch_front(gm_plan* p, const Batch& b, HeavyBatchState<V>* hs,
   tm.begin(PhaseTimes::kExpand, st);
   {
     const unsigned grid = static_cast<unsigned>((b.elems + kExpandTile - 1) / kExpandTile);
-    k4_expand<V><<<grid, kExpandThreads, 0, st>>>(p->seg_off, p->seg_bstart, p->seg_j, 0, p->n_seg,
+    k_tile_bounds<<<grid_for(grid, 256, p->num_sms), 256, 0, st>>>(p->seg_off, p->n_seg, b.elem0, b.elems, kExpandTile,
+                                                                 p->tile_meta);
+    ++p->stats.launches;
+    k4_expand<V><<<grid, kExpandThreads, 0, st>>>(p->seg_off, p->seg_bstart, p->seg_j, p->tile_meta,
                                                   static_cast<const V*>(p->A.vals), p->B.col_idx,
                                                   static_cast<const V*>(p->B.vals), b.elem0, b.elems, p->stage_col[0],
                                                   static_cast<V*>(p->stage_val[0]));
@@ -532,8 +538,10 @@ static int heavy_batch_front(gm_plan* p, const Batch& b, HeavyBatchState<V>* hs,
     const V* xv = static_cast<const V*>(p->stage_val[cur]);
     tm.begin(PhaseTimes::kHist, st);
     GM_CUDA(cudaMemsetAsync(p->counts, 0, static_cast<size_t>(n_child) * sizeof(u32), st));
+    k_tile_bounds<<<grid_for(grid, 256, p->num_sms), 256, 0, st>>>(off_cur, n_par, 0, b.elems, kSplitTile, p->tile_meta);
+    ++p->stats.launches;
     k5_level<V, false><<<grid, kSplitThreads, split_smem_bytes<V>(false), st>>>(
-        xc, xv, b.elems, off_cur, n_par, F, prm.shift[l], p->counts, nullptr, nullptr, nullptr);
+        xc, xv, b.elems, off_cur, n_par, p->tile_meta, F, prm.shift[l], p->counts, nullptr, nullptr, nullptr);
     ++p->stats.launches;
     GM_CUDA(cudaGetLastError());
     tm.end(st);
@@ -543,7 +551,7 @@ static int heavy_batch_front(gm_plan* p, const Batch& b, HeavyBatchState<V>* hs,
     tm.end(st);
     tm.begin(PhaseTimes::kSplit, st);
     k5_level<V, true><<<grid, kSplitThreads, split_smem_bytes<V>(true), st>>>(
-        xc, xv, b.elems, off_cur, n_par, F, prm.shift[l], nullptr, p->cursor, p->stage_col[cur ^ 1],
+        xc, xv, b.elems, off_cur, n_par, p->tile_meta, F, prm.shift[l], nullptr, p->cursor, p->stage_col[cur ^ 1],
         static_cast<V*>(p->stage_val[cur ^ 1]));
     ++p->stats.launches;
     GM_CUDA(cudaGetLastError());
@@ -945,5 +953,13 @@ const char* gm_status_string(int status) {
 }
 
 const char* gm_last_error(void) { return g_last_error.c_str(); }
+
+#ifdef GM_K6_PROFILE
+int gm_debug_k6_profile(unsigned long long* out16, int reset) {
+  cudaMemcpyFromSymbol(out16, g_k6_prof, 16 * sizeof(unsigned long long));
+  if (reset) { unsigned long long z[16] = {0}; cudaMemcpyToSymbol(g_k6_prof, z, sizeof(z)); }
+  return 0;
+}
+#endif
 
 }  // extern "C"

@@ -2,6 +2,7 @@
 #pragma once
 #include <cuda_runtime.h>
 
+#include <climits>
 #include <cstdint>
 
 namespace gm {
@@ -78,5 +79,34 @@ __device__ __forceinline__ i64 last_le(const T* __restrict__ a, i64 lo, i64 hi, 
 __device__ __forceinline__ int clamp_rel(i64 v, int lo, int hi) {
   return v < lo ? lo : (v > hi ? hi : static_cast<int>(v));
 }
+
+// What a tile-per-block kernel needs to know about the groups (rows, parents, segments) its tile touches.
+struct __align__(16) TileMeta {
+  i64 first;  // group that contains the tile's first element
+  int n;      // groups touched, first .. first + n - 1 (empty ones in between included)
+  int off1;   // start of group first + 1 relative to the tile (tile + 1 if n == 1)
+};
+
+// For every tile of `tile` consecutive elements (positions bias + t*tile ... of a flattened space whose
+// groups start at off[0..n_off)): the TileMeta above.  Run as its own small launch so that the searches of
+// all tiles overlap; a block that searched for its own tile would keep all its threads waiting through ~20
+// dependent global loads, and with this record the common tile (one or two groups) needs a single load.
+__global__ void k_tile_bounds(const i64* __restrict__ off, i64 n_off, i64 bias, i64 n_elems, int tile,
+                              TileMeta* __restrict__ meta) {
+  const i64 n_tiles = (n_elems + tile - 1) / tile;
+  for (i64 t = static_cast<i64>(blockIdx.x) * blockDim.x + threadIdx.x; t < n_tiles;
+       t += static_cast<i64>(gridDim.x) * blockDim.x) {
+    const i64 p0 = bias + t * tile;
+    const i64 p1 = bias + min(n_elems, (t + 1) * tile) - 1;
+    const i64 f = last_le(off, 0, n_off - 1, p0);
+    const i64 l = last_le(off, f, n_off - 1, p1);
+    TileMeta m;
+    m.first = f;
+    m.n = static_cast<int>(min(l - f + 1, static_cast<i64>(INT_MAX)));
+    m.off1 = m.n >= 2 ? clamp_rel(off[f + 1] - p0, -1, tile + 1) : tile + 1;
+    meta[t] = m;
+  }
+}
+
 
 }  // namespace gm

@@ -21,11 +21,10 @@ constexpr int kExpandUnroll = 4;
 template <typename V>
 __global__ void __launch_bounds__(kExpandThreads) k4_expand(
     const i64* __restrict__ seg_off, const i64* __restrict__ seg_bstart, const i64* __restrict__ seg_j,
-    i64 seg_lo_all, i64 seg_hi_all,   // segments of this batch: [seg_lo_all, seg_hi_all)
+    const TileMeta* __restrict__ tile_meta,  // per tile: first segment and number of segments
     const V* __restrict__ a_val, const int32_t* __restrict__ b_col, const V* __restrict__ b_val,
     i64 elem0, i64 n_elems,           // first product of the batch (global heavy numbering), batch size
     int32_t* __restrict__ x_col, V* __restrict__ x_val) {
-  __shared__ i64 s_range[2];
   __shared__ int s_rel[kExpandSegCap + 1];
   __shared__ i64 s_bstart[kExpandSegCap];
   __shared__ V s_aval[kExpandSegCap];
@@ -33,13 +32,9 @@ __global__ void __launch_bounds__(kExpandThreads) k4_expand(
   const i64 t0 = static_cast<i64>(blockIdx.x) * kExpandTile;
   const int tn = static_cast<int>(min(static_cast<i64>(kExpandTile), n_elems - t0));
   const i64 p0 = elem0 + t0;  // global product index of the tile's first element
-  if (threadIdx.x < 2) {
-    const i64 p = threadIdx.x == 0 ? p0 : p0 + tn - 1;
-    s_range[threadIdx.x] = last_le(seg_off, seg_lo_all, seg_hi_all - 1, p);
-  }
-  __syncthreads();
-  const i64 s_lo = s_range[0];
-  const i64 n_seg = s_range[1] - s_lo + 1;
+  const TileMeta tm = tile_meta[blockIdx.x];
+  const i64 s_lo = tm.first;
+  const i64 n_seg = tm.n;
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   constexpr int kPerWarp = kExpandTile / (kExpandThreads / 32);
   const int w0 = warp * kPerWarp;
@@ -97,7 +92,7 @@ __global__ void __launch_bounds__(kExpandThreads) k4_expand(
     // slow path: more segments than the shared table holds (very short rows of B): search per element
     for (int q = threadIdx.x; q < tn; q += kExpandThreads) {
       const i64 p = p0 + q;
-      const i64 s = last_le(seg_off, s_lo, s_range[1], p);
+      const i64 s = last_le(seg_off, s_lo, s_lo + n_seg - 1, p);
       const i64 src = seg_bstart[s] + (p - seg_off[s]);
       x_col[t0 + q] = b_col[src];
       x_val[t0 + q] = a_val[seg_j[s]] * b_val[src];

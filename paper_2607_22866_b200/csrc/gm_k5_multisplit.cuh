@@ -22,11 +22,14 @@
 
 namespace gm {
 
-constexpr int kSplitThreads = 512;
+#ifndef GM_SPLIT_THREADS
+#define GM_SPLIT_THREADS 512
+#endif
+constexpr int kSplitThreads = GM_SPLIT_THREADS;
 constexpr int kSplitItems = 16;
 constexpr int kSplitTile = kSplitThreads * kSplitItems;  // 8192 elements per block
-constexpr int kSplitBinCap = 2048;                       // bins (parent, child) per tile in shared memory
-constexpr int kSplitParentCap = 256;                     // parents per tile on the fast path
+constexpr int kSplitBinCap = 4 * kSplitThreads;           // bins (parent, child) per tile in shared memory
+constexpr int kSplitParentCap = kSplitThreads / 2;        // parents per tile on the fast path
 
 template <typename V>
 constexpr size_t split_smem_bytes(bool multisplit) {
@@ -42,9 +45,9 @@ struct SplitTileInfo {
 };
 
 template <typename V, bool MULTISPLIT>
-__global__ void __launch_bounds__(kSplitThreads, 2) k5_level(
+__global__ void __launch_bounds__(kSplitThreads, 1024 / kSplitThreads) k5_level(
     const int32_t* __restrict__ x_col, const V* __restrict__ x_val, i64 n_elems,
-    const i64* __restrict__ parent_off, i64 n_parents, int F, int shift,
+    const i64* __restrict__ parent_off, i64 n_parents, const TileMeta* __restrict__ tile_meta, int F, int shift,
     u32* __restrict__ counts,     // histogram: (n_parents * F) counters, zero-initialised
     u64* __restrict__ cursor,     // multisplit: (n_parents * F) write cursors, start = child_off
     int32_t* __restrict__ y_col, V* __restrict__ y_val) {
@@ -55,24 +58,32 @@ __global__ void __launch_bounds__(kSplitThreads, 2) k5_level(
   V* s_val = reinterpret_cast<V*>(s_pstart + kSplitParentCap + 15);  // aligned below
   s_val = reinterpret_cast<V*>((reinterpret_cast<uintptr_t>(s_val)) & ~uintptr_t{15});
   int32_t* s_col = reinterpret_cast<int32_t*>(s_val + kSplitTile);
-  __shared__ i64 s_range[2];
   __shared__ u32 s_scan[33];
 
   const i64 t0 = static_cast<i64>(blockIdx.x) * kSplitTile;
   const int tn = static_cast<int>(min(static_cast<i64>(kSplitTile), n_elems - t0));
   const int tid = threadIdx.x;
-  if (tid < 2) s_range[tid] = last_le(parent_off, 0, n_parents - 1, tid == 0 ? t0 : t0 + tn - 1);
-  __syncthreads();
-  const i64 p_lo = s_range[0];
-  const i64 n_par64 = s_range[1] - p_lo + 1;
+  const u32 lane = tid & 31;
+  // The tile's columns do not depend on any metadata: issue their loads first so that the metadata round
+  // trips below (tile bounds, then parent offsets) overlap with them instead of preceding them.
+  int32_t col[kSplitItems];
+#pragma unroll
+  for (int k = 0; k < kSplitItems; ++k) {
+    const int q = k * kSplitThreads + tid;
+    col[k] = q < tn ? x_col[t0 + q] : 0;
+  }
+  const TileMeta tm = tile_meta[blockIdx.x];  // same address for every thread: one broadcast load
+#pragma unroll
+  for (int k = 0; k < kSplitBinCap / kSplitThreads; ++k) s_bin[k * kSplitThreads + tid] = 0;
+  const i64 p_lo = tm.first;
   const u32 fmask = static_cast<u32>(F - 1);
 
-  if (n_par64 > kSplitParentCap || n_par64 * F > kSplitBinCap) {
+  if (tm.n > kSplitParentCap || static_cast<i64>(tm.n) * F > kSplitBinCap) {
     // ---- slow path: one global atomic per element
     for (int q = tid; q < tn; q += kSplitThreads) {
       const i64 p = t0 + q;
-      const i64 par = last_le(parent_off, p_lo, s_range[1], p);
-      const int32_t c = x_col[p];
+      const i64 par = last_le(parent_off, p_lo, p_lo + tm.n - 1, p);
+      const int32_t c = x_col[p];  // (the hoisted registers are striped differently; this path is rare)
       const i64 gbin = par * F + ((static_cast<u32>(c) >> shift) & fmask);
       if (MULTISPLIT) {
         const u64 dst = atomicAdd(&cursor[gbin], 1ull);
@@ -84,15 +95,17 @@ __global__ void __launch_bounds__(kSplitThreads, 2) k5_level(
     }
     return;
   }
-  const int n_par = static_cast<int>(n_par64);
+  const int n_par = tm.n;
   const int n_bins = n_par * F;
-  for (int b = tid; b < n_bins; b += kSplitThreads) s_bin[b] = 0;
-  for (int k = tid; k <= n_par; k += kSplitThreads)
-    s_poff[k] = (k == n_par) ? tn + 1 : clamp_rel(parent_off[p_lo + k] - t0, -1, tn + 1);
+  int bin_bits = 0;
+  while ((1 << bin_bits) < n_bins) ++bin_bits;
+  // one or two parents (the usual tile): the boundary came with the tile record; more: stage their offsets
+  if (n_par > 2)
+    for (int k = tid; k <= n_par; k += kSplitThreads)
+      s_poff[k] = (k == n_par) ? tn + 1 : clamp_rel(parent_off[p_lo + k] - t0, -1, tn + 1);
   __syncthreads();
 
   // ---- local histogram; every element learns its rank inside its bin
-  int32_t col[kSplitItems];
   u32 rank_bin[kSplitItems];  // (rank << 11) | bin
   static_assert(kSplitBinCap <= 2048 && kSplitTile <= (1 << 21), "rank/bin packing");
 #pragma unroll
@@ -100,9 +113,8 @@ __global__ void __launch_bounds__(kSplitThreads, 2) k5_level(
     const int q = k * kSplitThreads + tid;
     u32 bin = 0xffffffffu;
     if (q < tn) {
-      col[k] = x_col[t0 + q];
-      int par = 0;
-      if (n_par > 1) {
+      int par = q >= tm.off1 ? 1 : 0;
+      if (n_par > 2) {
         int lo = 0, hi = n_par - 1;
         while (lo < hi) {
           const int mid = lo + ((hi - lo + 1) >> 1);
@@ -112,10 +124,29 @@ __global__ void __launch_bounds__(kSplitThreads, 2) k5_level(
       }
       bin = static_cast<u32>(par * F) + ((static_cast<u32>(col[k]) >> shift) & fmask);
     }
-    // native shared-memory integer atomics run at ~12 per clock per SM on B200 whatever the skew; a warp
-    // match (match.any) to pre-aggregate equal bins measured 25x slower, so every element adds itself
+    // Rank inside the bin.  A shared-memory atomic that returns its old value costs one wavefront per lane
+    // that hits the same address, and with few bins (or one hot child) that is every lane.  So the lanes of a
+    // warp first find their peers in the same bin with one ballot per bin bit (the hardware match.any
+    // instruction measured 25x slower than this on B200), the lowest peer adds the group's size once, and
+    // every member takes base + its position among the peers.
     u32 rank = 0;
-    if (bin != 0xffffffffu) rank = atomicAdd(&s_bin[bin], 1u);
+    if (MULTISPLIT) {
+      u32 peers = 0xffffffffu;
+#pragma unroll 1
+      for (int b = 0; b < bin_bits; ++b) {
+        const bool bit = (bin >> b) & 1u;
+        const u32 bal = __ballot_sync(0xffffffffu, bit);
+        peers &= bit ? bal : ~bal;
+      }
+      peers &= __ballot_sync(0xffffffffu, bin != 0xffffffffu);
+      const int leader = __ffs(peers) - 1;
+      u32 base = 0;
+      if (bin != 0xffffffffu && static_cast<int>(lane) == leader) base = atomicAdd(&s_bin[bin], static_cast<u32>(__popc(peers)));
+      base = __shfl_sync(0xffffffffu, base, leader < 0 ? 0 : leader);
+      rank = base + __popc(peers & lanemask_lt());
+    } else {
+      if (bin != 0xffffffffu) atomicAdd(&s_bin[bin], 1u);
+    }
     rank_bin[k] = (rank << 11) | (bin & 2047u);
   }
   __syncthreads();

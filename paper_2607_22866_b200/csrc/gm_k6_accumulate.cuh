@@ -19,8 +19,8 @@
 
 namespace gm {
 
-constexpr int kAccTile = 2048;          // elements per ring stage
-constexpr int kAccMetaCap = 1024;       // chunk offsets / bases staged per refill
+// A block of BT threads streams tiles of 2 * BT products (two per thread) and keeps the offsets of BT chunks
+// at a time in shared memory.
 constexpr i64 kAccSegment = i64{1} << 18;  // elements per ticket
 constexpr int kAccSpinLimit = 1 << 24;  // polls of an mbarrier before the kernel gives up
 
@@ -50,19 +50,19 @@ __device__ __forceinline__ void bulk_g2s(void* dst, const void* src, u32 bytes, 
                : "memory");
 }
 
-// Number of ring stages that fit next to the accumulator.
-__host__ __device__ inline int acc_ring_stages(size_t smem_budget, int W, int val_bytes, bool numeric) {
+// Number of ring stages that fit next to the accumulator of a block of `bt` threads.
+__host__ __device__ inline int acc_ring_stages(size_t smem_budget, int W, int val_bytes, bool numeric, int bt) {
   const size_t fixed = static_cast<size_t>(W / 32) * 8 + (numeric ? static_cast<size_t>(W) * val_bytes : 0) +
-                       static_cast<size_t>(kAccMetaCap) * (4 + (numeric ? 8 : 0)) + 256;
-  const size_t stage = static_cast<size_t>(kAccTile) * (4 + (numeric ? val_bytes : 0));
+                       static_cast<size_t>(bt) * (4 + (numeric ? 8 : 0)) + 256;
+  const size_t stage = static_cast<size_t>(2 * bt) * (4 + (numeric ? val_bytes : 0));
   if (smem_budget <= fixed) return 0;
   size_t s = (smem_budget - fixed) / stage;
   return static_cast<int>(s > 8 ? 8 : s);
 }
-__host__ __device__ inline size_t acc_stream_smem_bytes(int W, int val_bytes, bool numeric, int stages) {
+__host__ __device__ inline size_t acc_stream_smem_bytes(int W, int val_bytes, bool numeric, int stages, int bt) {
   return static_cast<size_t>(W / 32) * 8 + (numeric ? static_cast<size_t>(W) * val_bytes : 0) +
-         static_cast<size_t>(kAccMetaCap) * (4 + (numeric ? 8 : 0)) +
-         static_cast<size_t>(stages) * kAccTile * (4 + (numeric ? val_bytes : 0)) + 256;
+         static_cast<size_t>(bt) * (4 + (numeric ? 8 : 0)) +
+         static_cast<size_t>(stages) * 2 * bt * (4 + (numeric ? val_bytes : 0)) + 256;
 }
 
 // seg_first[s] = first chunk whose start offset is >= s * kAccSegment (s = 0..n_segs); for the numeric
@@ -111,6 +111,8 @@ __global__ void __launch_bounds__(BT) k6_accumulate(
     const i64* __restrict__ chunk_base,          // numeric in: position in C of the chunk's first entry
     int32_t* __restrict__ c_col, V* __restrict__ c_val, i64 c_capacity, int* __restrict__ err) {
   extern __shared__ __align__(128) unsigned char smem_acc_raw[];
+  constexpr int kAccTile = 2 * BT;
+  constexpr int kAccMetaCap = BT;
   const int n_words = W >> 5;
   // layout: [ring cols][ring vals][acc][bitmap][meta base (i64)][meta off (i32)]
   int32_t* r_col = reinterpret_cast<int32_t*>(smem_acc_raw);
