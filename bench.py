@@ -147,8 +147,8 @@ def kernel_table(info, stats_avg, sv, nnz_b, n_light_entries_a):
         "k4_expand": (se * e + se * nnz_b + 24 * info.nnz_a_heavy, stats_avg["ms_expand"]),
         "k5a_histogram": (hist, stats_avg["ms_histogram"]),
         "k5b_multisplit": (split, stats_avg["ms_multisplit"]),
-        "k6_accumulate_symbolic": (4 * e + 12 * chunks, stats_avg["ms_acc_symbolic"]),
-        "k6_accumulate_numeric": (se * e + se * nnz_ch + 24 * chunks, stats_avg["ms_acc_numeric"]),
+        "k6_accumulate": (se * e + se * nnz_ch + 12 * chunks, stats_avg["ms_accumulate"]),
+        "k7_gather": (2 * se * nnz_ch + 24 * chunks, stats_avg["ms_gather"]),
     }
     return {k: {"bytes": int(b), "ms": float(ms), "gbs": (b / ms / 1e6 if ms > 0 else 0.0)} for k, (b, ms) in tbl.items()}
 
@@ -274,8 +274,8 @@ def main():
     dom = max(kt, key=lambda k: kt[k]["ms"])
     n_b = max(int(info.n_batches), 1)
     per_launch = {"k4_expand": n_b, "k5a_histogram": n_b * max(info.params.n_levels, 1),
-                  "k5b_multisplit": n_b * max(info.params.n_levels, 1), "k6_accumulate_symbolic": n_b,
-                  "k6_accumulate_numeric": n_b}.get(dom, 1)
+                  "k5b_multisplit": n_b * max(info.params.n_levels, 1), "k6_accumulate": n_b,
+                  "k7_gather": n_b}.get(dom, 1)
     roofline = {"kernel": dom, "bound": "hbm", "achieved": kt[dom]["gbs"], "peak": peak, "unit": "GB/s",
                 "frac": kt[dom]["gbs"] / peak, "peak_kind": f"of {peak_kind}", "traffic": None,
                 "bytes_per_launch": kt[dom]["bytes"] / per_launch, "ms_per_launch": kt[dom]["ms"] / per_launch,

@@ -118,7 +118,7 @@ typedef struct gm_exec_stats {
   int64_t final_chunks;        /* (row, chunk) pairs handed to the accumulate kernel           */
   int64_t launches;            /* kernels launched by this execute                             */
   float ms_light_symbolic, ms_light_numeric, ms_expand, ms_histogram, ms_multisplit,
-      ms_acc_symbolic, ms_acc_numeric, ms_scan, ms_total;
+      ms_accumulate, ms_gather, ms_scan, ms_total;
   float reserved[5];
 } gm_exec_stats;
 
@@ -166,8 +166,9 @@ int gm_spgemm_plan_ex(const gm_csr* A, const gm_csr* B, size_t smem_bytes,
 
 /* The rest of Algorithm 3: light rows by Gustavson's method with a shared-memory hash accumulator
  * (symbolic, then numeric); heavy rows, batch by batch, through the expansion (outer-product)
- * kernel (Algorithm 4), one histogram + multisplit (Algorithm 5) per level and the dense
- * chunk-accumulate kernel; C.row_ptr by prefix sums over the per-row counts.
+ * kernel (Algorithm 4), one histogram + multisplit (Algorithm 5) per level, the dense
+ * chunk-accumulate kernel (which compacts every chunk in place and counts its entries) and, once
+ * C.row_ptr is known by prefix sums over the per-row counts, the gather of the chunks into C.
  *   C_out  host struct filled with device pointers allocated through the allocator hook;
  *          C_out->nnz is exact.  Release with gm_csr_free.
  * Work is enqueued on `cuda_stream` (and internal streams forked from and joined back to it); the

@@ -71,7 +71,7 @@ class ExecStats(ctypes.Structure):
                 ("final_chunks", ctypes.c_int64), ("launches", ctypes.c_int64),
                 ("ms_light_symbolic", ctypes.c_float), ("ms_light_numeric", ctypes.c_float),
                 ("ms_expand", ctypes.c_float), ("ms_histogram", ctypes.c_float), ("ms_multisplit", ctypes.c_float),
-                ("ms_acc_symbolic", ctypes.c_float), ("ms_acc_numeric", ctypes.c_float), ("ms_scan", ctypes.c_float),
+                ("ms_accumulate", ctypes.c_float), ("ms_gather", ctypes.c_float), ("ms_scan", ctypes.c_float),
                 ("ms_total", ctypes.c_float), ("reserved", ctypes.c_float * 5)]
 
 

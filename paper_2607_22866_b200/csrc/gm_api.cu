@@ -14,6 +14,7 @@
 #include "gm_k4_expand.cuh"
 #include "gm_k5_multisplit.cuh"
 #include "gm_k6_accumulate.cuh"
+#include "gm_k7_gather.cuh"
 #include "gm_planner.h"
 #include "gm_scan.cuh"
 #include "gmagnus.h"
@@ -376,7 +377,7 @@ static int build_plan(gm_plan* p, cudaStream_t st) {
     GM_TRY(plan_alloc(p, &p->chunk_base, n_chunks_max + 1, st));
     GM_TRY(plan_alloc(p, &p->seg_first, static_cast<size_t>(info.stage_elems / kAccSegment) + 4, st));
     GM_TRY(plan_alloc(p, &p->ticket, 4, st));
-    const size_t n_tiles_max = static_cast<size_t>(info.stage_elems) / std::min(kExpandTile, kSplitTile) + 2;
+    const size_t n_tiles_max = static_cast<size_t>(info.stage_elems) / std::min({kExpandTile, kSplitTile, kGatherTile}) + 2;
     GM_TRY(plan_alloc(p, &p->tile_meta, n_tiles_max, st));
     int64_t* tmp2 = nullptr;  // the per-batch scans can be longer than the ones above
     GM_TRY(plan_alloc(p, &tmp2, static_cast<size_t>(scan_tmp_elems(std::max<i64>({static_cast<i64>(n_chunks_max), nnzA, nA, 1}))), st));
@@ -449,44 +450,38 @@ __global__ void k_rebase(const i64* __restrict__ in, i64 n, i64 bias, i64* __res
 
 template <typename V>
 struct HeavyBatchState {
-  const int32_t* fin_col = nullptr;  // staging buffer that holds the final chunks
-  const V* fin_val = nullptr;
+  int32_t* fin_col = nullptr;  // staging buffer that holds the final chunks
+  V* fin_val = nullptr;
   const i64* chunk_off = nullptr;    // n_chunks + 1 batch-relative offsets
   i64 n_chunks = 0;
   int log2_cpr = 0;
 };
 
-template <typename V, bool NUMERIC>
-static int launch_accumulate(gm_plan* p, const Batch& b, const HeavyBatchState<V>& hs, const i64* c_row_ptr,
-                             int32_t* c_col, V* c_val, i64 c_capacity, cudaStream_t st) {
+// K6: accumulate every chunk of the batch and compact it in place; chunk_nnz receives the entry counts.
+template <typename V>
+static int launch_accumulate(gm_plan* p, const Batch& b, const HeavyBatchState<V>& hs, cudaStream_t st) {
   const gm_params& prm = p->info.params;
   const int W = prm.chunk_width;
   const int ctas = prm.acc_ctas_per_sm;
   const size_t budget = p->smem_bytes / static_cast<size_t>(ctas) - 1024;
   const int bt = prm.acc_block_threads;
-  const int stages = acc_ring_stages(budget, W, sizeof(V), NUMERIC, bt);
+  const int stages = acc_ring_stages(budget, W, sizeof(V), true, bt);
   if (stages < 2) return fail(GM_ERR_UNSUPPORTED_SMEM, "shared memory budget too small for the accumulate kernel");
-  const size_t smem = acc_stream_smem_bytes(W, sizeof(V), NUMERIC, stages, bt);
+  const size_t smem = acc_stream_smem_bytes(W, sizeof(V), true, stages, bt);
   const i64 n_segs = (b.elems + kAccSegment - 1) / kAccSegment;
-  const i64 prep = std::max<i64>(n_segs + 1, NUMERIC ? hs.n_chunks : 0);
-  k6_prepare<<<static_cast<unsigned>((prep + 255) / 256), 256, 0, st>>>(
-      hs.chunk_off, hs.n_chunks, n_segs, p->seg_first, p->chunk_nnz_off, hs.log2_cpr, p->x_heavy, b.h0, c_row_ptr,
-      NUMERIC ? p->chunk_base : nullptr);
+  k6_prepare<<<static_cast<unsigned>((n_segs + 1 + 255) / 256), 256, 0, st>>>(hs.chunk_off, hs.n_chunks, n_segs, p->seg_first);
   GM_CUDA(cudaMemsetAsync(p->ticket, 0, sizeof(int), st));
-  if (!NUMERIC) GM_CUDA(cudaMemsetAsync(p->chunk_nnz, 0, static_cast<size_t>(hs.n_chunks) * sizeof(u32), st));
-  // symbolic launches keep only a bitmap next to the ring, so two blocks share an SM
-  const int per_sm = (NUMERIC ? 1024 : 2048) / bt;  // a symbolic block needs no value array: twice as many fit
+  GM_CUDA(cudaMemsetAsync(p->chunk_nnz, 0, static_cast<size_t>(hs.n_chunks) * sizeof(u32), st));
+  const int per_sm = 1024 / bt;
   const unsigned grid = static_cast<unsigned>(std::min<i64>(n_segs, static_cast<i64>(p->num_sms) * per_sm));
-#define GM_ACC(BT)                                                                                                    \
-  do {                                                                                                                \
-    auto kern = k6_accumulate<V, NUMERIC, BT>;                                                                        \
-    if (smem > 48 * 1024)                                                                                             \
-      GM_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)));      \
+#define GM_ACC(BT)                                                                                                   \
+  do {                                                                                                               \
+    auto kern = k6_accumulate<V, true, BT>;                                                                          \
+    if (smem > 48 * 1024)                                                                                            \
+      GM_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)));     \
     kern<<<grid, BT, smem, st>>>(hs.fin_col, hs.fin_val, hs.chunk_off, hs.n_chunks, p->seg_first, n_segs, p->ticket, \
-                                 hs.log2_cpr, W, stages, p->chunk_nnz, p->chunk_base, c_col, c_val, c_capacity,       \
-                                 p->err);                                                                             \
+                                 hs.log2_cpr, W, stages, p->chunk_nnz, p->err);                                      \
   } while (0)
-  // 1024 threads per SM in total: the floating-point shared-memory atomics are latency bound
   if (bt == 1024) GM_ACC(1024);
   else if (bt == 512) GM_ACC(512);
   else if (bt == 256) GM_ACC(256);
@@ -497,7 +492,24 @@ static int launch_accumulate(gm_plan* p, const Batch& b, const HeavyBatchState<V
   return GM_OK;
 }
 
-// Expansion, every multisplit level and the symbolic accumulate of one batch.  Leaves C^_reord in
+// K7: once C.rowPtr covers the batch's rows, move the compacted chunks into C.
+template <typename V>
+static int launch_gather(gm_plan* p, const Batch& b, const HeavyBatchState<V>& hs, const i64* c_row_ptr,
+                         int32_t* c_col, V* c_val, i64 c_capacity, cudaStream_t st) {
+  k6_chunk_bases<<<grid_for(hs.n_chunks, 256, p->num_sms), 256, 0, st>>>(p->chunk_nnz_off, hs.n_chunks, hs.log2_cpr,
+                                                                         p->x_heavy, b.h0, c_row_ptr, p->chunk_base);
+  // the batch's heavy entry count is only known on the device: it is at most the batch's product count
+  const unsigned grid = static_cast<unsigned>((b.elems + kGatherTile - 1) / kGatherTile);
+  k_tile_bounds<<<grid_for(grid, 256, p->num_sms), 256, 0, st>>>(p->chunk_nnz_off, hs.n_chunks, 0, 0, kGatherTile,
+                                                               p->tile_meta, p->chunk_nnz_off + hs.n_chunks);
+  k7_gather<V><<<grid, kGatherThreads, 0, st>>>(hs.fin_col, hs.fin_val, hs.chunk_off, p->chunk_nnz_off, p->chunk_base,
+                                                hs.n_chunks, p->tile_meta, c_col, c_val, c_capacity, p->err);
+  p->stats.launches += 3;
+  GM_CUDA(cudaGetLastError());
+  return GM_OK;
+}
+
+// Expansion, every multisplit level and the accumulate of one batch.  Leaves the compacted chunks in
 // the staging buffer and the per-chunk entry counts (and their scan) in chunk_nnz / chunk_nnz_off,
 // and writes the heavy rows' entry counts into row_nnz.
 template <typename V>
@@ -561,15 +573,15 @@ static int heavy_batch_front(gm_plan* p, const Batch& b, HeavyBatchState<V>* hs,
     n_par = n_child;
   }
   hs->fin_col = p->stage_col[cur];
-  hs->fin_val = static_cast<const V*>(p->stage_val[cur]);
+  hs->fin_val = static_cast<V*>(p->stage_val[cur]);
   hs->chunk_off = off_cur;
   hs->n_chunks = n_par;
   hs->log2_cpr = ilog2_floor(static_cast<uint64_t>(prm.chunks_required));
   p->stats.final_chunks += n_par;
   p->stats.staged_products += b.elems;
 
-  tm.begin(PhaseTimes::kAccSym, st);
-  GM_TRY((launch_accumulate<V, false>(p, b, *hs, nullptr, nullptr, nullptr, 0, st)));
+  tm.begin(PhaseTimes::kAccNum, st);
+  GM_TRY((launch_accumulate<V>(p, b, *hs, st)));
   tm.end(st);
   tm.begin(PhaseTimes::kScan, st);
   exclusive_scan<u32, i64>(p->chunk_nnz, p->chunk_nnz_off, hs->n_chunks, p->scan_tmp, nullptr, nullptr, nullptr, st);
@@ -666,8 +678,8 @@ static int execute_t(gm_plan* p, cudaStream_t st, gm_csr* C) {
     c_val = static_cast<V*>(dev_alloc(static_cast<size_t>(std::max<i64>(total, 1)) * sizeof(V), st));
     if (!c_col || !c_val) { cleanup(); return fail(GM_ERR_OOM, "allocation of C (" + std::to_string(total) + " entries) failed"); }
     if (n_batches == 1) {
-      tm.begin(PhaseTimes::kAccNum, st);
-      GM_TRY_C((launch_accumulate<V, true>(p, p->batches[0], hs, c_row_ptr, c_col, c_val, capacity, st)));
+      tm.begin(PhaseTimes::kAccSym, st);
+      GM_TRY_C((launch_gather<V>(p, p->batches[0], hs, c_row_ptr, c_col, c_val, capacity, st)));
       tm.end(st);
     }
     GM_TRY_C(light_numeric(capacity));
@@ -712,8 +724,8 @@ static int execute_t(gm_plan* p, cudaStream_t st, gm_csr* C) {
       exclusive_scan<int32_t, i64>(p->row_nnz + r0, c_row_ptr + r0, r1 - r0, p->scan_tmp, p->c_total, p->c_total, nullptr, st);
       p->stats.launches += 3;
       tm.end(st);
-      tm.begin(PhaseTimes::kAccNum, st);
-      GM_TRY_C((launch_accumulate<V, true>(p, b, hs, c_row_ptr, c_col, c_val, capacity, st)));
+      tm.begin(PhaseTimes::kAccSym, st);
+      GM_TRY_C((launch_gather<V>(p, b, hs, c_row_ptr, c_col, c_val, capacity, st)));
       tm.end(st);
     }
     GM_TRY_C(light_numeric(capacity));
@@ -747,8 +759,8 @@ static int execute_t(gm_plan* p, cudaStream_t st, gm_csr* C) {
     p->stats.ms_expand = ph[PhaseTimes::kExpand];
     p->stats.ms_histogram = ph[PhaseTimes::kHist];
     p->stats.ms_multisplit = ph[PhaseTimes::kSplit];
-    p->stats.ms_acc_symbolic = ph[PhaseTimes::kAccSym];
-    p->stats.ms_acc_numeric = ph[PhaseTimes::kAccNum];
+    p->stats.ms_gather = ph[PhaseTimes::kAccSym];
+    p->stats.ms_accumulate = ph[PhaseTimes::kAccNum];
     p->stats.ms_scan = ph[PhaseTimes::kScan];
     cudaEventElapsedTime(&p->stats.ms_total, ev_total0, ev_total1);
   }

@@ -92,7 +92,8 @@ struct __align__(16) TileMeta {
 // all tiles overlap; a block that searched for its own tile would keep all its threads waiting through ~20
 // dependent global loads, and with this record the common tile (one or two groups) needs a single load.
 __global__ void k_tile_bounds(const i64* __restrict__ off, i64 n_off, i64 bias, i64 n_elems, int tile,
-                              TileMeta* __restrict__ meta) {
+                              TileMeta* __restrict__ meta, const i64* __restrict__ n_elems_dev = nullptr) {
+  if (n_elems_dev) n_elems = *n_elems_dev;  // size only known on the device (then the grid covers an upper bound)
   const i64 n_tiles = (n_elems + tile - 1) / tile;
   for (i64 t = static_cast<i64>(blockIdx.x) * blockDim.x + threadIdx.x; t < n_tiles;
        t += static_cast<i64>(gridDim.x) * blockDim.x) {

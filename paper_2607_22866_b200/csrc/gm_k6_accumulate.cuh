@@ -3,9 +3,13 @@
 // [c*W, (c+1)*W), so its products are summed into a W-entry dense accumulator in shared memory; a
 // bitmap records which columns received a product (structural zeros are kept), a block-wide prefix
 // sum over the bitmap words gives every occupied column its rank, and the chunk is written to C in
-// ascending column order at   C.rowPtr[row] + (entries of the row's earlier chunks) + rank.
-//   symbolic launch: bitmap only -> entries per chunk (feeds C.rowPtr)
-//   numeric launch : values + bitmap -> C.col / C.val
+// ascending column order.
+//
+// One pass, no symbolic twin: the position of a chunk in C is only known once every earlier chunk has been
+// counted, so the kernel writes the compacted chunk *in place*, over the start of the chunk's own (already
+// consumed) products in the staging buffer — the output of a chunk never has more entries than its input —
+// and reports the entry count.  A prefix sum over those counts gives C.rowPtr, and the gather kernel below
+// moves the compacted chunks to   C.rowPtr[row] + (entries of the row's earlier chunks).
 //
 // B200 design.  The chunks of a batch lie back to back in the staging buffer, so the kernel does
 // not fetch chunk by chunk: the element space is cut into equal segments (static flattened
@@ -19,8 +23,10 @@
 
 namespace gm {
 
-// A block of BT threads streams tiles of 2 * BT products (two per thread) and keeps the offsets of BT chunks
-// at a time in shared memory.
+// A block of BT threads streams tiles of kAccPerThread * BT products and keeps the offsets of half as many
+// chunks at a time in shared memory.  Few threads with several products each: the per-tile and per-chunk
+// control code is executed by every warp, so a wide block multiplies it.
+constexpr int kAccPerThread = 2;
 constexpr i64 kAccSegment = i64{1} << 18;  // elements per ticket
 constexpr int kAccSpinLimit = 1 << 24;  // polls of an mbarrier before the kernel gives up
 
@@ -52,25 +58,21 @@ __device__ __forceinline__ void bulk_g2s(void* dst, const void* src, u32 bytes, 
 
 // Number of ring stages that fit next to the accumulator of a block of `bt` threads.
 __host__ __device__ inline int acc_ring_stages(size_t smem_budget, int W, int val_bytes, bool numeric, int bt) {
-  const size_t fixed = static_cast<size_t>(W / 32) * 8 + (numeric ? static_cast<size_t>(W) * val_bytes : 0) +
-                       static_cast<size_t>(bt) * (4 + (numeric ? 8 : 0)) + 256;
-  const size_t stage = static_cast<size_t>(2 * bt) * (4 + (numeric ? val_bytes : 0));
+  const size_t fixed = static_cast<size_t>(W / 32) * 12 + (numeric ? static_cast<size_t>(W) * val_bytes : 0) +
+                       static_cast<size_t>(kAccPerThread / 2 * bt) * 4 + 256;
+  const size_t stage = static_cast<size_t>(kAccPerThread * bt) * (4 + (numeric ? val_bytes : 0));
   if (smem_budget <= fixed) return 0;
   size_t s = (smem_budget - fixed) / stage;
   return static_cast<int>(s > 8 ? 8 : s);
 }
 __host__ __device__ inline size_t acc_stream_smem_bytes(int W, int val_bytes, bool numeric, int stages, int bt) {
-  return static_cast<size_t>(W / 32) * 8 + (numeric ? static_cast<size_t>(W) * val_bytes : 0) +
-         static_cast<size_t>(bt) * (4 + (numeric ? 8 : 0)) +
-         static_cast<size_t>(stages) * 2 * bt * (4 + (numeric ? val_bytes : 0)) + 256;
+  return static_cast<size_t>(W / 32) * 12 + (numeric ? static_cast<size_t>(W) * val_bytes : 0) +
+         static_cast<size_t>(kAccPerThread / 2 * bt) * 4 +
+         static_cast<size_t>(stages) * kAccPerThread * bt * (4 + (numeric ? val_bytes : 0)) + 256;
 }
 
-// seg_first[s] = first chunk whose start offset is >= s * kAccSegment (s = 0..n_segs); for the numeric
-// pass also the position in C of every chunk's first entry.
-__global__ void k6_prepare(const i64* __restrict__ chunk_off, i64 n_chunks, i64 n_segs, i64* __restrict__ seg_first,
-                           const i64* __restrict__ chunk_nnz_off, int log2_chunks_per_row,
-                           const int32_t* __restrict__ x_heavy, i64 h0, const i64* __restrict__ c_row_ptr,
-                           i64* __restrict__ chunk_base) {
+// seg_first[s] = first chunk whose start offset is >= s * kAccSegment (s = 0..n_segs).
+__global__ void k6_prepare(const i64* __restrict__ chunk_off, i64 n_chunks, i64 n_segs, i64* __restrict__ seg_first) {
   const i64 i = static_cast<i64>(blockIdx.x) * blockDim.x + threadIdx.x;
   if (i <= n_segs) {
     const i64 target = i * kAccSegment;
@@ -81,7 +83,14 @@ __global__ void k6_prepare(const i64* __restrict__ chunk_off, i64 n_chunks, i64 
     }
     seg_first[i] = lo;
   }
-  if (chunk_base && i < n_chunks) {
+}
+
+// Position in C of every chunk's first entry, once C.rowPtr of the batch's rows is known.
+__global__ void k6_chunk_bases(const i64* __restrict__ chunk_nnz_off, i64 n_chunks, int log2_chunks_per_row,
+                               const int32_t* __restrict__ x_heavy, i64 h0, const i64* __restrict__ c_row_ptr,
+                               i64* __restrict__ chunk_base) {
+  for (i64 i = static_cast<i64>(blockIdx.x) * blockDim.x + threadIdx.x; i < n_chunks;
+       i += static_cast<i64>(gridDim.x) * blockDim.x) {
     const i64 r = i >> log2_chunks_per_row;
     chunk_base[i] = c_row_ptr[x_heavy[h0 + r]] + (chunk_nnz_off[i] - chunk_nnz_off[r << log2_chunks_per_row]);
   }
@@ -103,16 +112,15 @@ __device__ __forceinline__ void acc_add(bool valid, u32 cl, V v, V* acc, u32* bi
 
 template <typename V, bool NUMERIC, int BT>
 __global__ void __launch_bounds__(BT) k6_accumulate(
-    const int32_t* __restrict__ x_col, const V* __restrict__ x_val,
+    int32_t* x_col, V* x_val,            // staging buffer: products in, compacted chunks out (in place)
     const i64* __restrict__ chunk_off,   // n_chunks + 1 batch-relative element offsets
     i64 n_chunks, const i64* __restrict__ seg_first, i64 n_segs, int* __restrict__ ticket,
     int log2_chunks_per_row, int W, int stages,
-    u32* __restrict__ chunk_nnz,                 // symbolic out (pre-zeroed: empty chunks are never visited)
-    const i64* __restrict__ chunk_base,          // numeric in: position in C of the chunk's first entry
-    int32_t* __restrict__ c_col, V* __restrict__ c_val, i64 c_capacity, int* __restrict__ err) {
+    u32* __restrict__ chunk_nnz,         // out, pre-zeroed: entries per chunk (empty chunks are never visited)
+    int* __restrict__ err) {
   extern __shared__ __align__(128) unsigned char smem_acc_raw[];
-  constexpr int kAccTile = 2 * BT;
-  constexpr int kAccMetaCap = BT;
+  constexpr int kAccTile = kAccPerThread * BT;
+  constexpr int kAccMetaCap = kAccTile / 2;
   const int n_words = W >> 5;
   // layout: [ring cols][ring vals][acc][bitmap][meta base (i64)][meta off (i32)]
   int32_t* r_col = reinterpret_cast<int32_t*>(smem_acc_raw);
@@ -120,12 +128,14 @@ __global__ void __launch_bounds__(BT) k6_accumulate(
   unsigned char* after_ring = smem_acc_raw + static_cast<size_t>(stages) * kAccTile * (4 + (NUMERIC ? sizeof(V) : 0));
   V* acc = reinterpret_cast<V*>(after_ring);
   u32* bitmap = reinterpret_cast<u32*>(after_ring + (NUMERIC ? static_cast<size_t>(W) * sizeof(V) : 0));
-  i64* m_base = reinterpret_cast<i64*>(bitmap + 2 * n_words);
-  int* m_off = reinterpret_cast<int*>(m_base + (NUMERIC ? kAccMetaCap : 0));
+  u32* word_prefix = bitmap + n_words;                                       // prefix of a dense word
+  unsigned short* dense_list = reinterpret_cast<unsigned short*>(word_prefix + n_words);  // n_words entries
+  int* m_off = reinterpret_cast<int*>(bitmap + 2 * n_words + ((n_words + 3) / 4) * 2);
   __shared__ u64 full_bar[8];
   __shared__ u32 s_scan[33];
   __shared__ i64 s_seg[2];
   __shared__ int s_abort;
+  __shared__ int s_dense_n;
 
   const int tid = threadIdx.x, lane = tid & 31;
   const u32 wmask = static_cast<u32>(W - 1);
@@ -142,6 +152,7 @@ __global__ void __launch_bounds__(BT) k6_accumulate(
   if (tid == 0) {
     for (int s = 0; s < stages; ++s) mbar_init(&full_bar[s], 1);
     s_abort = 0;
+    s_dense_n = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   __syncthreads();
@@ -181,7 +192,6 @@ __global__ void __launch_bounds__(BT) k6_accumulate(
       for (int i = tid; i < kAccMetaCap; i += BT) {
         const i64 kk = m0 + i;
         if (kk <= k_end) m_off[i] = static_cast<int>(chunk_off[kk] - lo_al);
-        if (NUMERIC && kk < k_end) m_base[i] = chunk_base[kk];
       }
     };
     load_meta();
@@ -252,52 +262,60 @@ __global__ void __launch_bounds__(BT) k6_accumulate(
           for (int i = 0; i < wpt; ++i) pc += __popc(bitmap[wb + i]);
         u32 total;
         u32 ex = block_exclusive_scan(pc, s_scan, &total);
-        if constexpr (!NUMERIC) {
-          if (wb < n_words)
-            for (int i = 0; i < wpt; ++i) bitmap[wb + i] = 0u;
-          if (tid == 0) chunk_nnz[m0 + kw] = total;
-        } else {
-          const i64 out0 = m_base[kw];
-          const bool fits = out0 + total <= c_capacity;
-          if (!fits && tid == 0) dev_set_error(err, kDevCapacity);
-          for (int i = 0; i < wpt; ++i) {
-            // words with few bits: their owner writes them; dense words: the whole warp writes one word at a time
-            u32 word = 0;
-            if (wb < n_words) word = bitmap[wb + i];
-            const u32 wpc = __popc(word);
-            const bool dense = wpc > 4;
-            if (wpc && !dense) {
-              u32 wbits = word;
-              i64 p = out0 + ex;
-              while (wbits) {
-                const int b = __ffs(wbits) - 1;
-                wbits &= wbits - 1;
-                const int slot = ((wb + i) << 5) + b;
-                if (fits) { c_col[p] = static_cast<int32_t>(col_base + slot); c_val[p] = acc[slot]; }
-                acc[slot] = V(0);
-                ++p;
-              }
-            }
-            u32 dmask = __ballot_sync(0xffffffffu, dense);
-            while (dmask) {
-              const int src = __ffs(dmask) - 1;
-              dmask &= dmask - 1;
-              const u32 wd = __shfl_sync(0xffffffffu, word, src);
-              const u32 wex = __shfl_sync(0xffffffffu, ex, src);
-              const int wi = __shfl_sync(0xffffffffu, wb + i, src);
-              if ((wd >> lane) & 1u) {
-                const int slot = (wi << 5) + lane;
-                if (fits) {
-                  const i64 p = out0 + wex + __popc(wd & lanemask_lt());
-                  c_col[p] = static_cast<int32_t>(col_base + slot);
-                  c_val[p] = acc[slot];
+        if (tid == 0) chunk_nnz[m0 + kw] = total;
+        {
+          // in place: the chunk's products [m_off[kw], ce) are all in shared memory or consumed by now
+          int32_t* const c_col = x_col + lo_al + m_off[kw];
+          V* const c_val = x_val + lo_al + m_off[kw];
+          constexpr i64 out0 = 0;
+          constexpr bool fits = true;
+          // Words with few bits are written by their owner.  Dense words cluster at the low end of the chunk
+          // (hub columns), i.e. in the first warps, so they go to a list that all warps then share out evenly;
+          // there the 32 lanes of a warp write one word at a time.
+          if (wb < n_words) {
+            for (int i = 0; i < wpt; ++i) {
+              const u32 word = bitmap[wb + i];
+              const u32 wpc = __popc(word);
+              if (wpc > 4) {
+                const int idx = atomicAdd(&s_dense_n, 1);
+                dense_list[idx] = static_cast<unsigned short>(wb + i);
+                word_prefix[wb + i] = ex;
+              } else if (wpc) {
+                u32 wbits = word;
+                i64 p = out0 + ex;
+                while (wbits) {
+                  const int b = __ffs(wbits) - 1;
+                  wbits &= wbits - 1;
+                  const int slot = ((wb + i) << 5) + b;
+                  if (fits) { c_col[p] = static_cast<int32_t>(col_base + slot); c_val[p] = acc[slot]; }
+                  acc[slot] = V(0);
+                  ++p;
                 }
-                acc[slot] = V(0);
+                bitmap[wb + i] = 0u;
               }
+              ex += wpc;
             }
-            if (wb < n_words) bitmap[wb + i] = 0u;
-            ex += wpc;
           }
+          __syncthreads();
+          const int n_dense = s_dense_n;
+          constexpr int kWarps = BT / 32;
+          for (int i = tid >> 5; i < n_dense; i += kWarps) {
+            const int wi = dense_list[i];
+            const u32 word = bitmap[wi];
+            if ((word >> lane) & 1u) {
+              const int slot = (wi << 5) + lane;
+              if (fits) {
+                const i64 p = out0 + word_prefix[wi] + __popc(word & lanemask_lt());
+                c_col[p] = static_cast<int32_t>(col_base + slot);
+                c_val[p] = acc[slot];
+              }
+              acc[slot] = V(0);
+            }
+            __syncwarp();
+            if (lane == 0) bitmap[wi] = 0u;
+          }
+          __syncthreads();
+          if (tid == 0) s_dense_n = 0;
         }
         __syncthreads();
         ++kw;
