@@ -95,11 +95,19 @@ def test_b200_defaults():
         raw = (s - n_min * (4 + sv) - 4) // (2 * (32 * 4 + 8))
         assert p.max_fanout == min(256, 1 << (raw.bit_length() - 1))
     assert p32.levels() == [32] and p64.levels() == [128]
-    # light-row capacity: table (<= 2 slots per entry) + 64-bit sort buffer must fit s_LM
+    # light-row capacity: table (<= 2 slots per entry) + 64-bit sort buffer must fit s_LM; the default
+    # threshold stops at 4096 products (beyond that the sort costs more than the heavy path), the
+    # capacity itself is 8192 and can be asked for, 16384 cannot
     for sv, p in ((4, p32), (8, p64)):
-        cap = 1 << (int(p.tau) - 1).bit_length()
-        assert p.light_slots * (4 + sv) + cap * 8 <= s and p.light_slots >= 1.5 * p.tau
-        assert 2 * cap * 8 + 3 * cap * (4 + sv) > s - 1024      # the next power of two would not fit
+        assert p.tau == 4096 and p.light_slots == 8192
+        dt = np.float32 if sv == 4 else np.float64
+        o = gm.PlanOpts(); o.tau = 8192
+        q = gm.planner_params(1 << 20, dt, s, o)
+        assert q.tau == 8192 and q.light_slots * (4 + sv) + 8192 * 8 <= s and q.light_slots >= 1.5 * 8192
+        assert 2 * 8192 * 8 + 3 * 8192 * (4 + sv) > s - 1024      # the next power of two would not fit
+        o.tau = 8193
+        with pytest.raises(gm.GmError):
+            gm.planner_params(1 << 20, dt, s, o)
     # wide column space: 2^24 columns -> 512 chunks -> two levels at the default fan-out
     p = gm.planner_params(1 << 24, np.float32, B200_SMEM)
     assert p.levels() == [256, 2]
