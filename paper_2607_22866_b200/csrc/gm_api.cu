@@ -473,6 +473,7 @@ static int launch_accumulate(gm_plan* p, const Batch& b, const HeavyBatchState<V
   GM_CUDA(cudaMemsetAsync(p->ticket, 0, sizeof(int), st));
   GM_CUDA(cudaMemsetAsync(p->chunk_nnz, 0, static_cast<size_t>(hs.n_chunks) * sizeof(u32), st));
   const int per_sm = 1024 / bt;
+  static const int small_max = [] { const char* e = std::getenv("GM_SMALL_CHUNK"); return e ? std::atoi(e) : kAccSmallChunk; }();
   const unsigned grid = static_cast<unsigned>(std::min<i64>(n_segs, static_cast<i64>(p->num_sms) * per_sm));
 #define GM_ACC(BT)                                                                                                   \
   do {                                                                                                               \
@@ -480,7 +481,7 @@ static int launch_accumulate(gm_plan* p, const Batch& b, const HeavyBatchState<V
     if (smem > 48 * 1024)                                                                                            \
       GM_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)));     \
     kern<<<grid, BT, smem, st>>>(hs.fin_col, hs.fin_val, hs.chunk_off, hs.n_chunks, p->seg_first, n_segs, p->ticket, \
-                                 hs.log2_cpr, W, stages, p->chunk_nnz, p->err);                                      \
+                                 hs.log2_cpr, W, stages, small_max, p->chunk_nnz, p->err);                                      \
   } while (0)
   if (bt == 1024) GM_ACC(1024);
   else if (bt == 512) GM_ACC(512);

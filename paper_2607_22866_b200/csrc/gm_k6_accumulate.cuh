@@ -110,12 +110,63 @@ __device__ __forceinline__ void acc_add(bool valid, u32 cl, V v, V* acc, u32* bi
   }
 }
 
+// Small chunks.  Going through the block-wide accumulator costs every chunk a few microseconds of barriers
+// and prefix sums whatever it holds, and most chunks of a power-law product hold few products.  A chunk of at
+// most kAccSmallChunk products that lies completely inside the current tile is instead handled by ONE warp,
+// with no block-wide step at all, so that 32 such chunks are in progress per block: the warp sorts the chunk's
+// (column, value) pairs in place in the shared-memory tile (bitonic network with ascending-only comparators,
+// so a length that is not a power of two needs no padding), adds up runs of equal columns and writes the
+// result over the chunk's start in the staging buffer.  This is the paper's separate branch for light chunks
+// (Section III-A), with a sort where the paper uses a hash table.
+constexpr int kAccSmallChunk = 32;
+
+template <typename V>
+__device__ __forceinline__ void small_chunk(int32_t* col, V* val, int n, int32_t* out_col, V* out_val,
+                                            u32* nnz_out) {
+  const int lane = threadIdx.x & 31;
+  int N = 1;
+  while (N < n) N <<= 1;
+  for (int k = 2; k <= N; k <<= 1) {
+    for (int j = k - 1, first = 1; j > 0; j = first ? (k >> 2) : (j >> 1), first = 0) {
+      for (int i = lane; i < n; i += 32) {
+        const int l = i ^ j;
+        if (l > i && l < n) {
+          const int32_t a = col[i], b = col[l];
+          if (a > b) {
+            col[i] = b; col[l] = a;
+            const V t = val[i]; val[i] = val[l]; val[l] = t;
+          }
+        }
+      }
+      __syncwarp();
+      if (first && k == 2) break;  // k = 2 has only the mirror step
+    }
+  }
+  // runs of equal columns: the lane that owns a run's first element adds the run up and writes it
+  int base = 0;
+  for (int b0 = 0; b0 < n; b0 += 32) {
+    const int i = b0 + lane;
+    const bool head = i < n && (i == 0 || col[i] != col[i - 1]);
+    const u32 heads = __ballot_sync(0xffffffffu, head);
+    if (head) {
+      const int32_t c = col[i];
+      V sum = val[i];
+      for (int q = i + 1; q < n && col[q] == c; ++q) sum += val[q];
+      const int p = base + __popc(heads & lanemask_lt());
+      out_col[p] = c;
+      out_val[p] = sum;
+    }
+    base += __popc(heads);
+  }
+  if (lane == 0) *nnz_out = static_cast<u32>(base);
+}
+
 template <typename V, bool NUMERIC, int BT>
-__global__ void __launch_bounds__(BT) k6_accumulate(
+__global__ void __launch_bounds__(BT, 1) k6_accumulate(
     int32_t* x_col, V* x_val,            // staging buffer: products in, compacted chunks out (in place)
     const i64* __restrict__ chunk_off,   // n_chunks + 1 batch-relative element offsets
     i64 n_chunks, const i64* __restrict__ seg_first, i64 n_segs, int* __restrict__ ticket,
-    int log2_chunks_per_row, int W, int stages,
+    int log2_chunks_per_row, int W, int stages, int small_max,
     u32* __restrict__ chunk_nnz,         // out, pre-zeroed: entries per chunk (empty chunks are never visited)
     int* __restrict__ err) {
   extern __shared__ __align__(128) unsigned char smem_acc_raw[];
@@ -215,16 +266,38 @@ __global__ void __launch_bounds__(BT) k6_accumulate(
       }
       const int tile_lo = j * kAccTile;
       const int tile_hi = min(end, tile_lo + kAccTile);
-      const int32_t* tc = r_col + st * kAccTile - tile_lo;
-      const V* tv = r_val + st * kAccTile - tile_lo;
+      int32_t* tc = r_col + st * kAccTile - tile_lo;
+      V* tv = r_val + st * kAccTile - tile_lo;
       while (pos < tile_hi) {
         // make sure the current chunk and its end are inside the metadata window
-        if (kw + 1 >= kAccMetaCap) {
+        if (kw + 33 >= kAccMetaCap) {  // the look-ahead below reads 32 chunks
           __syncthreads();
           m0 += kw;
           kw = 0;
           load_meta();
           __syncthreads();
+        }
+        if (pos == m_off[kw] && m_off[kw + 1] - pos <= small_max && m_off[kw + 1] <= tile_hi) {
+          // at the start of a small chunk: how many of the next 32 chunks are small and end inside this tile?  Every warp
+          // evaluates the same shared-memory metadata, so the answer is uniform without a barrier.
+          const i64 kc = m0 + kw + lane;
+          bool small = false;
+          if (kc < k_end) {
+            const int cs = m_off[kw + lane], cend = m_off[kw + lane + 1];
+            small = cend <= tile_hi && cend - cs <= small_max;
+          }
+          const u32 not_small = ~__ballot_sync(0xffffffffu, small);
+          const int run = not_small ? __ffs(not_small) - 1 : 32;
+          if (run > 0) {
+            const int w = tid >> 5;
+            if (w < run && !s_abort) {
+              const int cs = m_off[kw + w], cn = m_off[kw + w + 1] - cs;
+              if (cn > 0) small_chunk<V>(tc + cs, tv + cs, cn, x_col + lo_al + cs, x_val + lo_al + cs, &chunk_nnz[m0 + kw + w]);
+            }
+            kw += run;
+            pos = m_off[kw];
+            continue;
+          }
         }
         const int ce = m_off[kw + 1];
         if (ce <= pos) { ++kw; continue; }  // empty chunk
