@@ -196,6 +196,31 @@ int gm_plan_set_timing(gm_plan* plan, int enable);
  * DEVICE array ip_out (n_rows int64), on `cuda_stream`. */
 int gm_plan_get_row_products(const gm_plan* plan, int64_t* ip_out_device, void* cuda_stream);
 
+/* Row analysis for callers that must not allocate.  The paper has no counterpart: this is a packaging
+ * variant of the row-analysis kernels behind gm_spgemm_plan.
+ *
+ * Some callers cannot let a library allocate device memory on their behalf: a service that hands a
+ * fixed memory budget to each component at start-up, code that runs between the begin and end of a
+ * latency-critical section where an allocation (which may synchronise the whole device) is not
+ * acceptable, or a host whose allocator is owned by another runtime.  For them this entry point
+ * computes IP_i = sum over stored entries j of A[i,:] of nnz(B[A.col[j],:]) for every row of A and
+ * allocates nothing: no cudaMalloc / cudaFree, no stream-ordered allocation, no allocator hook.
+ * Its scratch (products per stored entry, their prefix sums, tile sums of the scan) lives in a
+ * fixed array inside the library image: about 12.6 MB of device memory on every GPU that loads the
+ * library, held until the process exits.
+ *   A, B           host structs with DEVICE pointers, as for gm_spgemm_plan (values are not read)
+ *   ip_out_device  DEVICE array of A->n_rows int64, written by the call
+ *   cuda_stream    the work is enqueued there; the call does not synchronise
+ * Limit: A->nnz <= GM_NOALLOC_MAX_NNZ_A (1,048,576); larger inputs are rejected with GM_ERR_CAPACITY
+ * and nothing is launched.  Any number of rows.
+ * The first call on each device looks up the address of the scratch array (one
+ * cudaGetSymbolAddress with that device current); make that first call before starting any stream
+ * capture.  Every call uses the same scratch array: everything in it is rewritten before it is
+ * read, so nothing needs clearing, but two calls whose kernels can overlap on the GPU (different
+ * streams, or concurrent host threads) race on it — serialise them. */
+#define GM_NOALLOC_MAX_NNZ_A 1048576
+int gm_row_products_noalloc(const gm_csr* A, const gm_csr* B, int64_t* ip_out_device, void* cuda_stream);
+
 /* Releases the arrays of a result produced by gm_spgemm_execute and zeroes the struct. */
 void gm_csr_free(gm_csr* C);
 void gm_plan_destroy(gm_plan* plan);

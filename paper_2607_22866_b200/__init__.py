@@ -11,6 +11,8 @@ from .binding import (  # noqa: F401
     planner_params,
     planner_batches,
     spgemm_plan,
+    row_products_noalloc,
+    NOALLOC_MAX_NNZ_A,
     spgemm_execute,
     spgemm,
     spgemm_host,

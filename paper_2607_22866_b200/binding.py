@@ -21,7 +21,7 @@ GM_MAX_LEVELS = 8
 EXPORTED_SYMBOLS = [
     "gm_set_allocator", "gm_planner_params", "gm_planner_batches", "gm_spgemm_plan", "gm_spgemm_plan_ex", "gm_spgemm_execute",
     "gm_spgemm_host", "gm_plan_get_info", "gm_exec_get_stats", "gm_plan_set_timing",
-    "gm_plan_get_row_products", "gm_csr_free", "gm_plan_destroy", "gm_status_string", "gm_last_error",
+    "gm_plan_get_row_products", "gm_row_products_noalloc", "gm_csr_free", "gm_plan_destroy", "gm_status_string", "gm_last_error",
 ]
 
 
@@ -120,6 +120,7 @@ def load_library(install_torch_allocator: bool = True):
         lib.gm_exec_get_stats.argtypes = [vp, P(ExecStats)]
         lib.gm_plan_set_timing.argtypes = [vp, ctypes.c_int]
         lib.gm_plan_get_row_products.argtypes = [vp, vp, vp]
+        lib.gm_row_products_noalloc.argtypes = [P(_CSR), P(_CSR), vp, vp]
         lib.gm_csr_free.argtypes = [P(_CSR)]
         lib.gm_csr_free.restype = None
         lib.gm_plan_destroy.argtypes = [vp]
@@ -232,6 +233,20 @@ class Plan:
             self.destroy()
         except Exception:
             pass
+
+
+NOALLOC_MAX_NNZ_A = 1048576
+
+
+def row_products_noalloc(A: DeviceCSR, B: DeviceCSR, out: torch.Tensor, stream=None) -> torch.Tensor:
+    """gm_row_products_noalloc: IP_i for every row of A, written into the caller's int64 device tensor
+    `out` (A.n_rows entries).  The library allocates nothing: its scratch is a fixed array in the library
+    image, so nnz(A) is limited to NOALLOC_MAX_NNZ_A and calls that overlap on the GPU race on it."""
+    assert out.dtype == torch.int64 and out.is_contiguous() and out.numel() >= A.n_rows
+    a, b = A._struct(), B._struct()
+    _check(load_library().gm_row_products_noalloc(ctypes.byref(a), ctypes.byref(b), out.data_ptr(),
+                                                  _stream_ptr(stream)), "gm_row_products_noalloc")
+    return out
 
 
 def spgemm_plan(A: DeviceCSR, B: DeviceCSR, smem_bytes: int = 232448, opts: PlanOpts | None = None,

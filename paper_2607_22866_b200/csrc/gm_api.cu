@@ -2,6 +2,7 @@
 // light and heavy paths, batching of the heavy rows and assembly of C.
 #include <algorithm>
 #include <climits>
+#include <cstddef>
 #include <cstdio>
 #include <cstdlib>
 #include <cstring>
@@ -976,3 +977,67 @@ int gm_debug_k6_profile(unsigned long long* out16, int reset) {
 #endif
 
 }  // extern "C"
+
+// ------------------------------------------------------------------------------------------------
+// Row analysis without any allocation (see gm_row_products_noalloc in gmagnus.h)
+// ------------------------------------------------------------------------------------------------
+namespace gm {
+
+constexpr i64 kNoAllocMaxNnz = GM_NOALLOC_MAX_NNZ_A;
+
+// Scratch of the no-allocation entry point, part of the library image on every device that loads it.
+// In host code this name is only a handle for cudaGetSymbolAddress, not a device address.
+struct NoAllocScratch {
+  i64 nz_off[kNoAllocMaxNnz + 8];                    // prefix sums of the products per stored entry of A
+  i64 scan_tmp[kNoAllocMaxNnz / kScanTile + 8];      // tile sums of the prefix sum
+  int32_t nz_len[kNoAllocMaxNnz + 8];                // products per stored entry of A
+};
+static __device__ __align__(256) NoAllocScratch g_noalloc_scratch;
+
+__global__ void k1_row_products_only(const i64* __restrict__ a_row_ptr, i64 n_rows, const i64* __restrict__ nz_off,
+                                     i64* __restrict__ ip) {
+  for (i64 i = static_cast<i64>(blockIdx.x) * blockDim.x + threadIdx.x; i < n_rows;
+       i += static_cast<i64>(gridDim.x) * blockDim.x)
+    ip[i] = nz_off[a_row_ptr[i + 1]] - nz_off[a_row_ptr[i]];
+}
+
+constexpr int kNoAllocMaxDevices = 64;
+static NoAllocScratch* g_noalloc_ptr[kNoAllocMaxDevices] = {nullptr};
+static int g_noalloc_sms[kNoAllocMaxDevices] = {0};
+
+}  // namespace gm
+
+extern "C" int gm_row_products_noalloc(const gm_csr* A, const gm_csr* B, int64_t* ip_out_device, void* cuda_stream) {
+  GM_TRY(check_csr_arg(A, "A"));
+  GM_TRY(check_csr_arg(B, "B"));
+  if (!ip_out_device && A->n_rows > 0) return fail(GM_ERR_INVALID_ARG, "ip_out_device is null");
+  if (A->n_cols != B->n_rows) return fail(GM_ERR_DIM_MISMATCH, "A.n_cols != B.n_rows");
+  if (A->nnz > kNoAllocMaxNnz)
+    return fail(GM_ERR_CAPACITY, "gm_row_products_noalloc handles at most " + std::to_string(kNoAllocMaxNnz) +
+                                     " stored entries of A (got " + std::to_string(A->nnz) + "): its scratch is a fixed array");
+  int dev = 0;
+  GM_CUDA(cudaGetDevice(&dev));
+  if (dev < 0 || dev >= kNoAllocMaxDevices) return fail(GM_ERR_INVALID_ARG, "device index out of range");
+  if (!g_noalloc_ptr[dev]) {
+    // set-up, once per device, with that device current: the device address behind the symbol
+    void* ptr = nullptr;
+    GM_CUDA(cudaGetSymbolAddress(&ptr, g_noalloc_scratch));
+    int sms = 0;
+    GM_CUDA(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
+    g_noalloc_sms[dev] = sms;
+    g_noalloc_ptr[dev] = static_cast<NoAllocScratch*>(ptr);
+  }
+  NoAllocScratch* sc = g_noalloc_ptr[dev];
+  const int sms = g_noalloc_sms[dev];
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  // scratch members are addressed through the device pointer, never through the host-side symbol
+  int32_t* nz_len = reinterpret_cast<int32_t*>(reinterpret_cast<char*>(sc) + offsetof(NoAllocScratch, nz_len));
+  i64* nz_off = reinterpret_cast<i64*>(reinterpret_cast<char*>(sc) + offsetof(NoAllocScratch, nz_off));
+  i64* scan_tmp = reinterpret_cast<i64*>(reinterpret_cast<char*>(sc) + offsetof(NoAllocScratch, scan_tmp));
+  if (A->nnz > 0) k1_nz_len<<<grid_for(A->nnz, 256, sms, 32), 256, 0, st>>>(A->col_idx, A->nnz, B->row_ptr, nz_len);
+  exclusive_scan<int32_t, i64>(nz_len, nz_off, A->nnz, scan_tmp, nullptr, nullptr, nullptr, st);
+  if (A->n_rows > 0)
+    k1_row_products_only<<<grid_for(A->n_rows, 256, sms), 256, 0, st>>>(A->row_ptr, A->n_rows, nz_off, ip_out_device);
+  GM_CUDA(cudaGetLastError());
+  return GM_OK;
+}
