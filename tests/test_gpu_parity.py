@@ -212,3 +212,50 @@ def test_host_entry_point():
     with pytest.raises(gm.GmError) as ei:
         gm.spgemm_host(A, B, rp, col[:5], val[:5])
     assert ei.value.status == -6
+
+
+def _check_sampled_rows(A, B, n_random=200, n_heavy=60, **opts):
+    """Full-size check in the launch configuration the benchmark times: structure and values of
+    sampled rows (random rows, the heaviest rows, random heavy rows) against the row-range oracle,
+    plus whole-matrix invariants that need no reference."""
+    from parity import TOL
+    C, info, stats = run_gpu(A, B, **opts)
+    ip = oracle.row_products(A, B)
+    assert info.products_total == int(ip.sum()) and info.rows_heavy == int((ip > info.params.tau).sum())
+    rp = C.row_ptr.cpu().numpy()
+    assert rp[0] == 0 and rp[-1] == C.nnz == stats.c_nnz and np.all(np.diff(rp) >= 0)
+    assert np.all(np.diff(rp) <= np.minimum(ip, B.n_cols)) and np.all((np.diff(rp) == 0) == (ip == 0))
+    rng = np.random.default_rng(0)
+    rows = set(rng.integers(0, A.n_rows, n_random).tolist()) | set(np.argsort(-ip)[:3].tolist())
+    heavy = np.nonzero(ip > info.params.tau)[0]
+    if heavy.size:
+        rows |= set(rng.choice(heavy, min(n_heavy, heavy.size), replace=False).tolist())
+    for r in sorted(rows):
+        ref = oracle.spgemm(A, B, r, r + 1, threads=1)
+        s, e = rp[r], rp[r + 1]
+        assert e - s == ref.nnz, r
+        assert np.array_equal(C.col[s:e].cpu().numpy(), ref.col), r
+        val = C.val[s:e].cpu().numpy().astype(np.float64)
+        assert np.all(np.abs(val - ref.val) <= TOL[np.dtype(A.val.dtype)] * ref.abs), r
+    return info, stats
+
+
+def test_config2_rmat20_full_size_sampled_rows():
+    # the benchmark's default workload: 2.1e10 products, 9.7e9 entries of C, dozens of batches
+    A, B, _ = gen.config_inputs(2)
+    info, stats = _check_sampled_rows(A, B)
+    assert info.n_batches > 10 and info.params.levels() == [32] and stats.c_capacity >= stats.c_nnz
+
+
+def test_config3_rmat_fp64_two_levels_sampled_rows():
+    # fp64 R-MAT (scale 18 here, scale 21 in the config) with the fan-out capped so that the split takes two levels
+    A, B, _ = gen.config_inputs(3, shrink=3)
+    info, stats = _check_sampled_rows(A, B, max_fanout=8, stage_elems=1 << 26)
+    assert info.params.n_levels == 2 and info.n_batches > 1
+
+
+def test_config4_zipf_wide_columns_three_levels_sampled_rows():
+    # rectangular clipped-Zipf product, 2^22 columns here (2^24 in the config), three multisplit levels
+    A, B, _ = gen.config_inputs(4, shrink=2)
+    info, stats = _check_sampled_rows(A, B, n_random=60, n_heavy=40, max_fanout=8, chunk_width=8192)
+    assert info.params.n_levels == 3 and info.rows_heavy > 0
