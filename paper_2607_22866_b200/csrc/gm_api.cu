@@ -167,6 +167,7 @@ struct gm_plan {
   int64_t* chunk_base = nullptr;   // numeric pass: position in C of every chunk's first entry
   int64_t* seg_first = nullptr;    // accumulate kernel: first chunk of every element segment
   int* ticket = nullptr;
+  gm::TileMeta* row_meta = nullptr;   // per tile of the expansion kernel: heavy rows it touches (fused histogram)
   gm::TileMeta* tile_meta = nullptr;  // per tile of the expansion / multisplit kernels: groups it touches
   gm::PhaseTimes times;
 };
@@ -380,6 +381,7 @@ static int build_plan(gm_plan* p, cudaStream_t st) {
     GM_TRY(plan_alloc(p, &p->ticket, 4, st));
     const size_t n_tiles_max = static_cast<size_t>(info.stage_elems) / std::min({kExpandTile, kSplitTile, kGatherTile}) + 2;
     GM_TRY(plan_alloc(p, &p->tile_meta, n_tiles_max, st));
+    GM_TRY(plan_alloc(p, &p->row_meta, n_tiles_max, st));
     int64_t* tmp2 = nullptr;  // the per-batch scans can be longer than the ones above
     GM_TRY(plan_alloc(p, &tmp2, static_cast<size_t>(scan_tmp_elems(std::max<i64>({static_cast<i64>(n_chunks_max), nnzA, nA, 1}))), st));
     p->scan_tmp = tmp2;
@@ -519,25 +521,34 @@ static int heavy_batch_front(gm_plan* p, const Batch& b, HeavyBatchState<V>* hs,
   const gm_params& prm = p->info.params;
   const i64 rows_b = b.h1 - b.h0;
   PhaseTimes& tm = p->times;
-  tm.begin(PhaseTimes::kExpand, st);
-  {
-    const unsigned grid = static_cast<unsigned>((b.elems + kExpandTile - 1) / kExpandTile);
-    k_tile_bounds<<<grid_for(grid, 256, p->num_sms), 256, 0, st>>>(p->seg_off, p->n_seg, b.elem0, b.elems, kExpandTile,
-                                                                 p->tile_meta);
-    ++p->stats.launches;
-    k4_expand<V><<<grid, kExpandThreads, 0, st>>>(p->seg_off, p->seg_bstart, p->seg_j, p->tile_meta,
-                                                  static_cast<const V*>(p->A.vals), p->B.col_idx,
-                                                  static_cast<const V*>(p->B.vals), b.elem0, b.elems, p->stage_col[0],
-                                                  static_cast<V*>(p->stage_val[0]));
-    ++p->stats.launches;
-    GM_CUDA(cudaGetLastError());
-  }
-  tm.end(st);
   // level-0 parents are the batch's rows: offsets relative to the batch
   i64* off_cur = p->level_off[0];
   i64* off_nxt = p->level_off[1];
   k_rebase<<<grid_for(rows_b + 1, 256, p->num_sms), 256, 0, st>>>(p->heavy_base + b.h0, rows_b + 1, b.elem0, off_cur);
   ++p->stats.launches;
+  // the expansion kernel counts the first level's (row, child) bins while it writes, unless asked not to
+  const bool fuse_hist = prm.n_levels > 0 && !p->opts.separate_histogram;
+  tm.begin(PhaseTimes::kExpand, st);
+  {
+    static_assert(kExpandTile == kSplitTile, "the fused histogram shares the multisplit's tiles");
+    const unsigned grid = static_cast<unsigned>((b.elems + kExpandTile - 1) / kExpandTile);
+    k_tile_bounds<<<grid_for(grid, 256, p->num_sms), 256, 0, st>>>(p->seg_off, p->n_seg, b.elem0, b.elems, kExpandTile,
+                                                                 p->tile_meta);
+    ++p->stats.launches;
+    if (fuse_hist) {
+      GM_CUDA(cudaMemsetAsync(p->counts, 0, static_cast<size_t>(rows_b) * prm.fanout[0] * sizeof(u32), st));
+      k_tile_bounds<<<grid_for(grid, 256, p->num_sms), 256, 0, st>>>(off_cur, rows_b, 0, b.elems, kExpandTile, p->row_meta);
+      ++p->stats.launches;
+    }
+    k4_expand<V><<<grid, kExpandThreads, 0, st>>>(p->seg_off, p->seg_bstart, p->seg_j, p->tile_meta,
+                                                  static_cast<const V*>(p->A.vals), p->B.col_idx,
+                                                  static_cast<const V*>(p->B.vals), b.elem0, b.elems, p->stage_col[0],
+                                                  static_cast<V*>(p->stage_val[0]), p->row_meta, off_cur,
+                                                  fuse_hist ? prm.fanout[0] : 0, fuse_hist ? prm.shift[0] : 0, p->counts);
+    ++p->stats.launches;
+    GM_CUDA(cudaGetLastError());
+  }
+  tm.end(st);
   int cur = 0;
   i64 n_par = rows_b;
   if (prm.n_levels > 0) {
@@ -551,13 +562,15 @@ static int heavy_batch_front(gm_plan* p, const Batch& b, HeavyBatchState<V>* hs,
     const int32_t* xc = p->stage_col[cur];
     const V* xv = static_cast<const V*>(p->stage_val[cur]);
     tm.begin(PhaseTimes::kHist, st);
-    GM_CUDA(cudaMemsetAsync(p->counts, 0, static_cast<size_t>(n_child) * sizeof(u32), st));
     k_tile_bounds<<<grid_for(grid, 256, p->num_sms), 256, 0, st>>>(off_cur, n_par, 0, b.elems, kSplitTile, p->tile_meta);
     ++p->stats.launches;
-    k5_level<V, false><<<grid, kSplitThreads, split_smem_bytes<V>(false), st>>>(
-        xc, xv, b.elems, off_cur, n_par, p->tile_meta, F, prm.shift[l], p->counts, nullptr, nullptr, nullptr);
-    ++p->stats.launches;
-    GM_CUDA(cudaGetLastError());
+    if (!(l == 0 && fuse_hist)) {
+      GM_CUDA(cudaMemsetAsync(p->counts, 0, static_cast<size_t>(n_child) * sizeof(u32), st));
+      k5_level<V, false><<<grid, kSplitThreads, split_smem_bytes<V>(false), st>>>(
+          xc, xv, b.elems, off_cur, n_par, p->tile_meta, F, prm.shift[l], p->counts, nullptr, nullptr, nullptr);
+      ++p->stats.launches;
+      GM_CUDA(cudaGetLastError());
+    }
     tm.end(st);
     tm.begin(PhaseTimes::kScan, st);
     exclusive_scan<u32, i64>(p->counts, off_nxt, n_child, p->scan_tmp, nullptr, nullptr, reinterpret_cast<i64*>(p->cursor), st);

@@ -8,6 +8,10 @@
 //     col = B.col[seg_bstart[s] + (p - seg_off[s])],  val = A.val[seg_j[s]] * B.val[...]
 // for the segment s that contains p (Eq. 3 with a division-free search).  Each warp walks a
 // contiguous part of the tile, so reads of B and writes of the staging buffer are coalesced runs.
+//
+// The kernel can also count, for the first multisplit level, how many of the products it writes fall
+// into each (row, child) bin — the Histogram step of Algorithm 3 — while the columns are still in
+// registers, which saves a pass over the staging buffer (4 bytes per product).
 #pragma once
 #include "gm_common.cuh"
 
@@ -17,6 +21,8 @@ constexpr int kExpandThreads = 256;
 constexpr int kExpandTile = 8192;     // products per block
 constexpr int kExpandSegCap = 1024;   // segments staged in shared memory; tiles with more take the slow path
 constexpr int kExpandUnroll = 4;
+constexpr int kExpandHistCap = 2048;      // (row, child) bins of the fused histogram kept in shared memory
+constexpr int kExpandHistParents = 256;
 
 template <typename V>
 __global__ void __launch_bounds__(kExpandThreads) k4_expand(
@@ -24,7 +30,12 @@ __global__ void __launch_bounds__(kExpandThreads) k4_expand(
     const TileMeta* __restrict__ tile_meta,  // per tile: first segment and number of segments
     const V* __restrict__ a_val, const int32_t* __restrict__ b_col, const V* __restrict__ b_val,
     i64 elem0, i64 n_elems,           // first product of the batch (global heavy numbering), batch size
-    int32_t* __restrict__ x_col, V* __restrict__ x_val) {
+    int32_t* __restrict__ x_col, V* __restrict__ x_val,
+    // fused level-0 histogram (hist_F == 0: off): rows of the batch as parents
+    const TileMeta* __restrict__ row_meta, const i64* __restrict__ row_off, int hist_F, int hist_shift,
+    u32* __restrict__ counts) {
+  __shared__ u32 s_hist[kExpandHistCap];
+  __shared__ int s_roff[kExpandHistParents + 1];
   __shared__ int s_rel[kExpandSegCap + 1];
   __shared__ i64 s_bstart[kExpandSegCap];
   __shared__ V s_aval[kExpandSegCap];
@@ -36,6 +47,41 @@ __global__ void __launch_bounds__(kExpandThreads) k4_expand(
   const i64 s_lo = tm.first;
   const i64 n_seg = tm.n;
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  // fused histogram set-up: hist_mode 0 = off, 1 = bins in shared memory, 2 = too many rows in the tile (global atomics)
+  int hist_mode = 0, h_npar = 1;
+  TileMeta rm{};
+  const u32 h_mask = static_cast<u32>(hist_F - 1);
+  if (hist_F > 0) {
+    rm = row_meta[blockIdx.x];
+    h_npar = rm.n;
+    hist_mode = (rm.n > kExpandHistParents || static_cast<i64>(rm.n) * hist_F > kExpandHistCap) ? 2 : 1;
+    if (hist_mode == 1) {
+      for (int b = threadIdx.x; b < rm.n * hist_F; b += kExpandThreads) s_hist[b] = 0;
+      if (rm.n > 2)
+        for (int k = threadIdx.x; k <= rm.n; k += kExpandThreads)
+          s_roff[k] = (k == rm.n) ? tn + 1 : clamp_rel(row_off[rm.first + k] - t0, -1, tn + 1);
+    }
+  }
+  if (hist_mode == 1) __syncthreads();  // bins zeroed before anybody counts (uniform: same record for all threads)
+  auto count_product = [&](int q, int32_t c) {
+    if (hist_mode == 0) return;
+    const u32 child = (static_cast<u32>(c) >> hist_shift) & h_mask;
+    if (hist_mode == 1) {
+      int par = q >= rm.off1 ? 1 : 0;
+      if (h_npar > 2) {
+        int lo = 0, hi = h_npar - 1;
+        while (lo < hi) {
+          const int mid = lo + ((hi - lo + 1) >> 1);
+          if (s_roff[mid] <= q) lo = mid; else hi = mid - 1;
+        }
+        par = lo;
+      }
+      atomicAdd(&s_hist[par * hist_F + child], 1u);
+    } else {
+      const i64 par = last_le(row_off, rm.first, rm.first + rm.n - 1, t0 + q);
+      atomicAdd(&counts[par * hist_F + child], 1u);
+    }
+  };
   constexpr int kPerWarp = kExpandTile / (kExpandThreads / 32);
   const int w0 = warp * kPerWarp;
   const int w1 = min(tn, w0 + kPerWarp);
@@ -50,7 +96,6 @@ __global__ void __launch_bounds__(kExpandThreads) k4_expand(
       }
     }
     __syncthreads();
-    if (w0 >= w1) return;
     // warp-uniform start: last segment whose start is <= w0 (zero-length segments are skipped by taking the last)
     int cur = 0;
     {
@@ -61,6 +106,7 @@ __global__ void __launch_bounds__(kExpandThreads) k4_expand(
       }
       cur = lo;
     }
+    if (w0 < w1)
     for (int q0 = w0; q0 < w1; q0 += 32 * kExpandUnroll) {
       int32_t col[kExpandUnroll];
       V val[kExpandUnroll], av[kExpandUnroll];
@@ -85,6 +131,7 @@ __global__ void __launch_bounds__(kExpandThreads) k4_expand(
         if (q < w1) {
           x_col[t0 + q] = col[u];
           x_val[t0 + q] = av[u] * val[u];
+          count_product(q, col[u]);
         }
       }
     }
@@ -94,8 +141,18 @@ __global__ void __launch_bounds__(kExpandThreads) k4_expand(
       const i64 p = p0 + q;
       const i64 s = last_le(seg_off, s_lo, s_lo + n_seg - 1, p);
       const i64 src = seg_bstart[s] + (p - seg_off[s]);
-      x_col[t0 + q] = b_col[src];
+      const int32_t c = b_col[src];
+      x_col[t0 + q] = c;
       x_val[t0 + q] = a_val[seg_j[s]] * b_val[src];
+      count_product(q, c);
+    }
+  }
+  if (hist_mode == 1) {
+    __syncthreads();
+    const i64 g0 = rm.first * hist_F;
+    for (int b = threadIdx.x; b < h_npar * hist_F; b += kExpandThreads) {
+      const u32 c = s_hist[b];
+      if (c) atomicAdd(&counts[g0 + b], c);
     }
   }
 }

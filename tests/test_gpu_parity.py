@@ -259,3 +259,12 @@ def test_config4_zipf_wide_columns_three_levels_sampled_rows():
     A, B, _ = gen.config_inputs(4, shrink=2)
     info, stats = _check_sampled_rows(A, B, n_random=60, n_heavy=40, max_fanout=8, chunk_width=8192)
     assert info.params.n_levels == 3 and info.rows_heavy > 0
+
+
+@pytest.mark.parametrize("separate", [0, 1])
+def test_fused_and_stand_alone_histogram_agree(separate):
+    # level-0 counts come either from the expansion kernel (default) or from the histogram kernel
+    A = gen.rmat(13, 16, seed=11, dtype=np.float32)
+    C, info, stats = check_product(A, A, tau=512, chunk_width=512, max_fanout=4, separate_histogram=separate,
+                                   stage_elems=1 << 20)
+    assert info.params.n_levels == 2 and info.n_batches > 1
