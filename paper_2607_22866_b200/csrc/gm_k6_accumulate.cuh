@@ -289,10 +289,11 @@ __global__ void __launch_bounds__(BT, 1) k6_accumulate(
           const u32 not_small = ~__ballot_sync(0xffffffffu, small);
           const int run = not_small ? __ffs(not_small) - 1 : 32;
           if (run > 0) {
-            const int w = tid >> 5;
-            if (w < run && !s_abort) {
-              const int cs = m_off[kw + w], cn = m_off[kw + w + 1] - cs;
-              if (cn > 0) small_chunk<V>(tc + cs, tv + cs, cn, x_col + lo_al + cs, x_val + lo_al + cs, &chunk_nnz[m0 + kw + w]);
+            if (!s_abort) {
+              for (int w = tid >> 5; w < run; w += BT / 32) {  // one chunk per warp, round-robin
+                const int cs = m_off[kw + w], cn = m_off[kw + w + 1] - cs;
+                if (cn > 0) small_chunk<V>(tc + cs, tv + cs, cn, x_col + lo_al + cs, x_val + lo_al + cs, &chunk_nnz[m0 + kw + w]);
+              }
             }
             kw += run;
             pos = m_off[kw];

@@ -268,3 +268,12 @@ def test_fused_and_stand_alone_histogram_agree(separate):
     C, info, stats = check_product(A, A, tau=512, chunk_width=512, max_fanout=4, separate_histogram=separate,
                                    stage_elems=1 << 20)
     assert info.params.n_levels == 2 and info.n_batches > 1
+
+
+@pytest.mark.parametrize("ctas", [1, 2, 4, 8])
+def test_accumulators_per_sm_with_many_tiny_chunks(ctas):
+    # narrow blocks (fewer warps than the 32-chunk look-ahead of the small-chunk path) and chunks of a few
+    # products each: every chunk must still be visited exactly once
+    A, B, _ = gen.config_inputs(4, shrink=4)
+    C, info, stats = check_product(A, B, acc_ctas_per_sm=ctas, tau=256)
+    assert info.rows_heavy > 100 and info.params.acc_ctas_per_sm == ctas
