@@ -36,6 +36,13 @@ SMEM_BYTES = 232448
 DEFAULT_CONFIG = 2  # R-MAT scale 20, edge factor 16, fp32: the largest fp32 power-law product
 
 
+# DRAM bytes per launch (ncu dram__bytes_read.sum + dram__bytes_write.sum) over the algorithmic bytes of the same
+# launch, measured on a scaled-down case of the same kernels (R-MAT scale 17, 134 M products per batch: see
+# profiles/dram_traffic_rmat17_f32.md).  Traffic grows in proportion to the products processed, so a full-size
+# launch is the algorithmic figure times this ratio.
+TRAFFIC_RATIO = {"k4_expand": 1.05, "k5b_multisplit": 1.03, "k6_accumulate": 1.00, "k7_gather": 1.08}
+
+
 def _peaks():
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(path):
@@ -277,7 +284,9 @@ def main():
                   "k5b_multisplit": n_b * max(info.params.n_levels, 1), "k6_accumulate": n_b,
                   "k7_gather": n_b}.get(dom, 1)
     roofline = {"kernel": dom, "bound": "hbm", "achieved": kt[dom]["gbs"], "peak": peak, "unit": "GB/s",
-                "frac": kt[dom]["gbs"] / peak, "peak_kind": f"of {peak_kind}", "traffic": None,
+                "frac": kt[dom]["gbs"] / peak, "peak_kind": f"of {peak_kind}",
+                "traffic": (kt[dom]["bytes"] / per_launch * TRAFFIC_RATIO[dom]) if dom in TRAFFIC_RATIO else None,
+                "traffic_source": "ncu on R-MAT scale 17, scaled by products (profiles/dram_traffic_rmat17_f32.md)",
                 "bytes_per_launch": kt[dom]["bytes"] / per_launch, "ms_per_launch": kt[dom]["ms"] / per_launch,
                 "launches_per_step": per_launch}
 

@@ -359,7 +359,7 @@ static int build_plan(gm_plan* p, cudaStream_t st) {
       p->max_batch_rows = std::max(p->max_batch_rows, b.h1 - b.h0);
     }
     // the accumulate kernel streams whole tiles: it may read (and ignore) up to one tile past the last product
-    const size_t se = static_cast<size_t>(info.stage_elems) + 2048 + 8;
+    const size_t se = static_cast<size_t>(info.stage_elems) + 4096 + 8;
     const int n_buf = prm.n_levels > 0 ? 2 : 1;
     for (int i = 0; i < n_buf; ++i) {
       GM_TRY(plan_alloc(p, &p->stage_col[i], se, st));
@@ -468,9 +468,16 @@ static int launch_accumulate(gm_plan* p, const Batch& b, const HeavyBatchState<V
   const int ctas = prm.acc_ctas_per_sm;
   const size_t budget = p->smem_bytes / static_cast<size_t>(ctas) - 1024;
   const int bt = prm.acc_block_threads;
-  const int stages = acc_ring_stages(budget, W, sizeof(V), true, bt);
+  // four products per thread and tile when two such stages fit next to the accumulator (the per-tile control
+  // code is executed by every warp, so bigger tiles amortise it), otherwise two
+  int pt = 4;
+  int stages = acc_ring_stages(budget, W, sizeof(V), true, bt, pt);
+  if (stages < 2) {
+    pt = 2;
+    stages = acc_ring_stages(budget, W, sizeof(V), true, bt, pt);
+  }
   if (stages < 2) return fail(GM_ERR_UNSUPPORTED_SMEM, "shared memory budget too small for the accumulate kernel");
-  const size_t smem = acc_stream_smem_bytes(W, sizeof(V), true, stages, bt);
+  const size_t smem = acc_stream_smem_bytes(W, sizeof(V), true, stages, bt, pt);
   const i64 n_segs = (b.elems + kAccSegment - 1) / kAccSegment;
   k6_prepare<<<static_cast<unsigned>((n_segs + 1 + 255) / 256), 256, 0, st>>>(hs.chunk_off, hs.n_chunks, n_segs, p->seg_first);
   GM_CUDA(cudaMemsetAsync(p->ticket, 0, sizeof(int), st));
@@ -478,19 +485,21 @@ static int launch_accumulate(gm_plan* p, const Batch& b, const HeavyBatchState<V
   const int per_sm = 1024 / bt;
   static const int small_max = [] { const char* e = std::getenv("GM_SMALL_CHUNK"); return e ? std::atoi(e) : kAccSmallChunk; }();
   const unsigned grid = static_cast<unsigned>(std::min<i64>(n_segs, static_cast<i64>(p->num_sms) * per_sm));
-#define GM_ACC(BT)                                                                                                   \
+#define GM_ACC2(BT, PT)                                                                                              \
   do {                                                                                                               \
-    auto kern = k6_accumulate<V, true, BT>;                                                                          \
+    auto kern = k6_accumulate<V, true, BT, PT>;                                                                      \
     if (smem > 48 * 1024)                                                                                            \
       GM_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)));     \
     kern<<<grid, BT, smem, st>>>(hs.fin_col, hs.fin_val, hs.chunk_off, hs.n_chunks, p->seg_first, n_segs, p->ticket, \
                                  hs.log2_cpr, W, stages, small_max, p->chunk_nnz, p->err);                                      \
   } while (0)
+#define GM_ACC(BT) do { if (pt == 4) GM_ACC2(BT, 4); else GM_ACC2(BT, 2); } while (0)
   if (bt == 1024) GM_ACC(1024);
   else if (bt == 512) GM_ACC(512);
   else if (bt == 256) GM_ACC(256);
   else GM_ACC(128);
 #undef GM_ACC
+#undef GM_ACC2
   p->stats.launches += 2;
   GM_CUDA(cudaGetLastError());
   return GM_OK;

@@ -23,10 +23,9 @@
 
 namespace gm {
 
-// A block of BT threads streams tiles of kAccPerThread * BT products and keeps the offsets of half as many
+// A block of BT threads streams tiles of PT * BT products (PT = 2 or 4 per thread) and keeps the offsets of BT
 // chunks at a time in shared memory.  Few threads with several products each: the per-tile and per-chunk
 // control code is executed by every warp, so a wide block multiplies it.
-constexpr int kAccPerThread = 2;
 constexpr i64 kAccSegment = i64{1} << 18;  // elements per ticket
 constexpr int kAccSpinLimit = 1 << 24;  // polls of an mbarrier before the kernel gives up
 
@@ -57,18 +56,18 @@ __device__ __forceinline__ void bulk_g2s(void* dst, const void* src, u32 bytes, 
 }
 
 // Number of ring stages that fit next to the accumulator of a block of `bt` threads.
-__host__ __device__ inline int acc_ring_stages(size_t smem_budget, int W, int val_bytes, bool numeric, int bt) {
+__host__ __device__ inline int acc_ring_stages(size_t smem_budget, int W, int val_bytes, bool numeric, int bt, int pt) {
   const size_t fixed = static_cast<size_t>(W / 32) * 12 + (numeric ? static_cast<size_t>(W) * val_bytes : 0) +
-                       static_cast<size_t>(kAccPerThread / 2 * bt) * 4 + 256;
-  const size_t stage = static_cast<size_t>(kAccPerThread * bt) * (4 + (numeric ? val_bytes : 0));
+                       static_cast<size_t>(bt) * 4 + 256;
+  const size_t stage = static_cast<size_t>(pt * bt) * (4 + (numeric ? val_bytes : 0));
   if (smem_budget <= fixed) return 0;
   size_t s = (smem_budget - fixed) / stage;
   return static_cast<int>(s > 8 ? 8 : s);
 }
-__host__ __device__ inline size_t acc_stream_smem_bytes(int W, int val_bytes, bool numeric, int stages, int bt) {
+__host__ __device__ inline size_t acc_stream_smem_bytes(int W, int val_bytes, bool numeric, int stages, int bt, int pt) {
   return static_cast<size_t>(W / 32) * 12 + (numeric ? static_cast<size_t>(W) * val_bytes : 0) +
-         static_cast<size_t>(kAccPerThread / 2 * bt) * 4 +
-         static_cast<size_t>(stages) * kAccPerThread * bt * (4 + (numeric ? val_bytes : 0)) + 256;
+         static_cast<size_t>(bt) * 4 +
+         static_cast<size_t>(stages) * pt * bt * (4 + (numeric ? val_bytes : 0)) + 256;
 }
 
 // seg_first[s] = first chunk whose start offset is >= s * kAccSegment (s = 0..n_segs).
@@ -161,7 +160,7 @@ __device__ __forceinline__ void small_chunk(int32_t* col, V* val, int n, int32_t
   if (lane == 0) *nnz_out = static_cast<u32>(base);
 }
 
-template <typename V, bool NUMERIC, int BT>
+template <typename V, bool NUMERIC, int BT, int PT>
 __global__ void __launch_bounds__(BT, 1) k6_accumulate(
     int32_t* x_col, V* x_val,            // staging buffer: products in, compacted chunks out (in place)
     const i64* __restrict__ chunk_off,   // n_chunks + 1 batch-relative element offsets
@@ -170,8 +169,8 @@ __global__ void __launch_bounds__(BT, 1) k6_accumulate(
     u32* __restrict__ chunk_nnz,         // out, pre-zeroed: entries per chunk (empty chunks are never visited)
     int* __restrict__ err) {
   extern __shared__ __align__(128) unsigned char smem_acc_raw[];
-  constexpr int kAccTile = kAccPerThread * BT;
-  constexpr int kAccMetaCap = kAccTile / 2;
+  constexpr int kAccTile = PT * BT;
+  constexpr int kAccMetaCap = BT;
   const int n_words = W >> 5;
   // layout: [ring cols][ring vals][acc][bitmap][meta base (i64)][meta off (i32)]
   int32_t* r_col = reinterpret_cast<int32_t*>(smem_acc_raw);
