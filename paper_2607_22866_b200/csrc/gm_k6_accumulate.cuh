@@ -238,6 +238,9 @@ __global__ void __launch_bounds__(BT, 1) k6_accumulate(
     // chunk metadata of the segment, refilled every kAccMetaCap chunks
     i64 m0 = k_first;          // first chunk held in the metadata window
     int kw = 0;                // current chunk = m0 + kw
+    const u32 crow_mask = (1u << log2_chunks_per_row) - 1u;
+    u32 crow = static_cast<u32>(k_first) & crow_mask;  // index of the current chunk inside its row (kept in step with kw)
+    const int log2W = 31 - __clz(W);
     auto load_meta = [&]() {
       for (int i = tid; i < kAccMetaCap; i += BT) {
         const i64 kk = m0 + i;
@@ -295,14 +298,15 @@ __global__ void __launch_bounds__(BT, 1) k6_accumulate(
               }
             }
             kw += run;
+            crow = (crow + static_cast<u32>(run)) & crow_mask;
             pos = m_off[kw];
             continue;
           }
         }
         const int ce = m_off[kw + 1];
-        if (ce <= pos) { ++kw; continue; }  // empty chunk
+        if (ce <= pos) { ++kw; crow = (crow + 1u) & crow_mask; continue; }  // empty chunk
         const int sub_hi = min(tile_hi, ce);
-        const u32 col_base = static_cast<u32>((m0 + kw) & ((i64{1} << log2_chunks_per_row) - 1)) * static_cast<u32>(W);
+        const u32 col_base = crow << log2W;
         if (!s_abort) {
           for (int base = pos; base < sub_hi; base += BT * kPerThread) {
             u32 cl[kPerThread];
@@ -319,7 +323,9 @@ __global__ void __launch_bounds__(BT, 1) k6_accumulate(
                 if (NUMERIC) v[u] = tv[q];
               }
               cl[u] = c & wmask;
+#ifdef GM_DEBUG_CHECKS
               if (c - cl[u] != col_base) { dev_set_error(err, kDevBadChunk); ok[u] = false; }
+#endif
             }
 #pragma unroll
             for (int u = 0; u < kPerThread; ++u) acc_add<V, NUMERIC>(ok[u], cl[u], v[u], acc, bitmap);
@@ -392,6 +398,7 @@ __global__ void __launch_bounds__(BT, 1) k6_accumulate(
         }
         __syncthreads();
         ++kw;
+        crow = (crow + 1u) & crow_mask;
       }
       // ---- the stage is free again: refill it
       __syncthreads();
