@@ -63,9 +63,8 @@ __global__ void __launch_bounds__(kExpandThreads) k4_expand(
     }
   }
   if (hist_mode == 1) __syncthreads();  // bins zeroed before anybody counts (uniform: same record for all threads)
-  auto count_product = [&](int q, int32_t c) {
-    if (hist_mode == 0) return;
-    const u32 child = (static_cast<u32>(c) >> hist_shift) & h_mask;
+  // row (parent) of tile position q, as an index into the tile's bins; -1 = global path
+  auto find_par = [&](int q) -> i64 {
     if (hist_mode == 1) {
       int par = q >= rm.off1 ? 1 : 0;
       if (h_npar > 2) {
@@ -76,11 +75,17 @@ __global__ void __launch_bounds__(kExpandThreads) k4_expand(
         }
         par = lo;
       }
-      atomicAdd(&s_hist[par * hist_F + child], 1u);
-    } else {
-      const i64 par = last_le(row_off, rm.first, rm.first + rm.n - 1, t0 + q);
-      atomicAdd(&counts[par * hist_F + child], 1u);
+      return par;
     }
+    return last_le(row_off, rm.first, rm.first + rm.n - 1, t0 + q);
+  };
+  auto count_in = [&](i64 par, int32_t c) {
+    const u32 child = (static_cast<u32>(c) >> hist_shift) & h_mask;
+    if (hist_mode == 1) atomicAdd(&s_hist[static_cast<int>(par) * hist_F + child], 1u);
+    else atomicAdd(&counts[par * hist_F + child], 1u);
+  };
+  auto count_product = [&](int q, int32_t c) {
+    if (hist_mode != 0) count_in(find_par(q), c);
   };
   constexpr int kPerWarp = kExpandTile / (kExpandThreads / 32);
   const int w0 = warp * kPerWarp;
@@ -110,6 +115,27 @@ __global__ void __launch_bounds__(kExpandThreads) k4_expand(
     for (int q0 = w0; q0 < w1; q0 += 32 * kExpandUnroll) {
       int32_t col[kExpandUnroll];
       V val[kExpandUnroll], av[kExpandUnroll];
+      // heavy rows mostly multiply long rows of B: when the next 32 * kExpandUnroll products all come from the
+      // segment the warp is in, nobody searches and the segment's data stays in uniform registers
+      while (q0 >= s_rel[cur + 1]) ++cur;  // uniform: cur is the same in every lane here
+      if (q0 + 32 * kExpandUnroll <= min(s_rel[cur + 1], w1)) {
+        const i64 src0 = s_bstart[cur] + (q0 - s_rel[cur]) + lane;
+        const V a = s_aval[cur];
+#pragma unroll
+        for (int u = 0; u < kExpandUnroll; ++u) {
+          col[u] = b_col[src0 + u * 32];
+          val[u] = b_val[src0 + u * 32];
+        }
+        const i64 par = hist_mode != 0 ? find_par(q0) : 0;  // a segment lies inside one row
+#pragma unroll
+        for (int u = 0; u < kExpandUnroll; ++u) {
+          const int q = q0 + u * 32 + lane;
+          x_col[t0 + q] = col[u];
+          x_val[t0 + q] = a * val[u];
+          if (hist_mode != 0) count_in(par, col[u]);
+        }
+        continue;
+      }
 #pragma unroll
       for (int u = 0; u < kExpandUnroll; ++u) {
         const int q = q0 + u * 32 + lane;
