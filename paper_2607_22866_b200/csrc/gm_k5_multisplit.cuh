@@ -131,19 +131,39 @@ __global__ void __launch_bounds__(kSplitThreads, 1024 / kSplitThreads) k5_level(
     // every member takes base + its position among the peers.
     u32 rank = 0;
     if (MULTISPLIT) {
-      u32 peers = 0xffffffffu;
+      // Products reach a parent in runs that come from one row of B, i.e. with ascending columns, so
+      // neighbouring lanes usually fall into the same bin.  A run of equal bins is found with one shuffle and
+      // one ballot; its first lane adds the run's length to the bin with one atomic and the members take
+      // base + their offset in the run.  Only when a warp has many short runs (columns in random order) are the
+      // peers of a bin matched across the whole warp, one ballot per bin bit, so that a hot bin still costs one
+      // atomic per warp and not one per lane.
+      const u32 prev = __shfl_up_sync(0xffffffffu, bin, 1);
+      const bool head = lane == 0 || bin != prev;
+      const u32 heads = __ballot_sync(0xffffffffu, head);
+      if (__popc(heads) <= 12) {
+        const u32 below = heads & (lanemask_lt() | (1u << lane));      // heads at or before this lane
+        const int start = 31 - __clz(below);                            // first lane of my run
+        const u32 above = heads & ~((2u << lane) - 1u);                 // heads after this lane
+        const int endl = above ? __ffs(above) - 1 : 32;                 // one past the last lane of my run
+        u32 base = 0;
+        if (head && bin != 0xffffffffu) base = atomicAdd(&s_bin[bin], static_cast<u32>(endl - start));
+        base = __shfl_sync(0xffffffffu, base, start);
+        rank = base + static_cast<u32>(lane - start);
+      } else {
+        u32 peers = 0xffffffffu;
 #pragma unroll 1
-      for (int b = 0; b < bin_bits; ++b) {
-        const bool bit = (bin >> b) & 1u;
-        const u32 bal = __ballot_sync(0xffffffffu, bit);
-        peers &= bit ? bal : ~bal;
+        for (int b = 0; b < bin_bits; ++b) {
+          const bool bit = (bin >> b) & 1u;
+          const u32 bal = __ballot_sync(0xffffffffu, bit);
+          peers &= bit ? bal : ~bal;
+        }
+        peers &= __ballot_sync(0xffffffffu, bin != 0xffffffffu);
+        const int leader = __ffs(peers) - 1;
+        u32 base = 0;
+        if (bin != 0xffffffffu && static_cast<int>(lane) == leader) base = atomicAdd(&s_bin[bin], static_cast<u32>(__popc(peers)));
+        base = __shfl_sync(0xffffffffu, base, leader < 0 ? 0 : leader);
+        rank = base + __popc(peers & lanemask_lt());
       }
-      peers &= __ballot_sync(0xffffffffu, bin != 0xffffffffu);
-      const int leader = __ffs(peers) - 1;
-      u32 base = 0;
-      if (bin != 0xffffffffu && static_cast<int>(lane) == leader) base = atomicAdd(&s_bin[bin], static_cast<u32>(__popc(peers)));
-      base = __shfl_sync(0xffffffffu, base, leader < 0 ? 0 : leader);
-      rank = base + __popc(peers & lanemask_lt());
     } else {
       if (bin != 0xffffffffu) atomicAdd(&s_bin[bin], 1u);
     }
@@ -214,12 +234,21 @@ __global__ void __launch_bounds__(kSplitThreads, 1024 / kSplitThreads) k5_level(
   __syncthreads();
 
   // ---- coalesced write: slot s belongs to the bin recomputed from its column and its parent
-  const u64 hi_base = 0;  // batch-relative positions fit 32 bits (checked by the planner)
-  (void)hi_base;
+  if (n_par == 1) {
+    // the usual tile (one parent): the bin is the child, nothing to search
+#pragma unroll 4
+    for (int s = tid; s < tn; s += kSplitThreads) {
+      const int32_t c = s_col[s];
+      const u32 dst = static_cast<u32>(s) + s_bin[(static_cast<u32>(c) >> shift) & fmask];
+      y_col[dst] = c;
+      y_val[dst] = s_val[s];
+    }
+    return;
+  }
   for (int s = tid; s < tn; s += kSplitThreads) {
     const int32_t c = s_col[s];
     int par = 0;
-    if (n_par > 1) {
+    {
       int lo = 0, hi = n_par - 1;
       while (lo < hi) {
         const int mid = lo + ((hi - lo + 1) >> 1);
