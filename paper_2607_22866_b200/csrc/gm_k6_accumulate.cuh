@@ -279,7 +279,8 @@ __global__ void __launch_bounds__(BT, 1) k6_accumulate(
           load_meta();
           __syncthreads();
         }
-        if (pos == m_off[kw] && m_off[kw + 1] - pos <= small_max && m_off[kw + 1] <= tile_hi) {
+        const int ce = m_off[kw + 1];
+        if (ce - pos <= small_max && ce <= tile_hi && pos == m_off[kw]) {
           // at the start of a small chunk: how many of the next 32 chunks are small and end inside this tile?  Every warp
           // evaluates the same shared-memory metadata, so the answer is uniform without a barrier.
           const i64 kc = m0 + kw + lane;
@@ -303,32 +304,32 @@ __global__ void __launch_bounds__(BT, 1) k6_accumulate(
             continue;
           }
         }
-        const int ce = m_off[kw + 1];
         if (ce <= pos) { ++kw; crow = (crow + 1u) & crow_mask; continue; }  // empty chunk
         const int sub_hi = min(tile_hi, ce);
         const u32 col_base = crow << log2W;
         if (!s_abort) {
           for (int base = pos; base < sub_hi; base += BT * kPerThread) {
-            u32 cl[kPerThread];
-            V v[kPerThread];
-            bool ok[kPerThread];
+            // slots of this warp that still hold products of the sub-range (warp-uniform): a short sub-range
+            // must not pay for the whole unrolled body
+            const int wq = base + (tid & ~31);
+            const int nu = wq >= sub_hi ? 0 : min(kPerThread, (sub_hi - wq + BT - 1) / BT);
+            if (nu == kPerThread && wq + (kPerThread - 1) * BT + 32 <= sub_hi) {
+              u32 cl[kPerThread];
+              V v[kPerThread];
 #pragma unroll
-            for (int u = 0; u < kPerThread; ++u) {
-              const int q = base + u * BT + tid;
-              ok[u] = q < sub_hi;
-              u32 c = col_base;
-              v[u] = V(0);
-              if (ok[u]) {
-                c = static_cast<u32>(tc[q]);
+              for (int u = 0; u < kPerThread; ++u) {
+                const int q = base + u * BT + tid;
+                cl[u] = static_cast<u32>(tc[q]) & wmask;
                 if (NUMERIC) v[u] = tv[q];
               }
-              cl[u] = c & wmask;
-#ifdef GM_DEBUG_CHECKS
-              if (c - cl[u] != col_base) { dev_set_error(err, kDevBadChunk); ok[u] = false; }
-#endif
-            }
 #pragma unroll
-            for (int u = 0; u < kPerThread; ++u) acc_add<V, NUMERIC>(ok[u], cl[u], v[u], acc, bitmap);
+              for (int u = 0; u < kPerThread; ++u) acc_add<V, NUMERIC>(true, cl[u], v[u], acc, bitmap);
+            } else {
+              for (int u = 0; u < nu; ++u) {
+                const int q = base + u * BT + tid;
+                if (q < sub_hi) acc_add<V, NUMERIC>(true, static_cast<u32>(tc[q]) & wmask, NUMERIC ? tv[q] : V(0), acc, bitmap);
+              }
+            }
           }
         }
         pos = sub_hi;
@@ -337,8 +338,12 @@ __global__ void __launch_bounds__(BT, 1) k6_accumulate(
         __syncthreads();
         const int wb = tid * wpt;
         u32 pc = 0;
-        if (wb < n_words)
-          for (int i = 0; i < wpt; ++i) pc += __popc(bitmap[wb + i]);
+        u32 word0 = 0;  // the thread's first (for wpt == 1: only) word stays in a register
+        if (wb < n_words) {
+          word0 = bitmap[wb];
+          pc = __popc(word0);
+          for (int i = 1; i < wpt; ++i) pc += __popc(bitmap[wb + i]);
+        }
         u32 total;
         u32 ex = block_exclusive_scan(pc, s_scan, &total);
         if (tid == 0) chunk_nnz[m0 + kw] = total;
@@ -353,7 +358,7 @@ __global__ void __launch_bounds__(BT, 1) k6_accumulate(
           // there the 32 lanes of a warp write one word at a time.
           if (wb < n_words) {
             for (int i = 0; i < wpt; ++i) {
-              const u32 word = bitmap[wb + i];
+              const u32 word = i == 0 ? word0 : bitmap[wb + i];
               const u32 wpc = __popc(word);
               if (wpc > 4) {
                 const int idx = atomicAdd(&s_dense_n, 1);
