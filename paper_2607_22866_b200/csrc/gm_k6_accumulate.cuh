@@ -185,7 +185,7 @@ __global__ void __launch_bounds__(BT, 1) k6_accumulate(
   __shared__ u32 s_scan[33];
   __shared__ i64 s_seg[2];
   __shared__ int s_abort;
-  __shared__ int s_dense_n;
+  __shared__ int s_dense_n[2];  // used by alternate chunks, so that resetting one needs no barrier of its own
 
   const int tid = threadIdx.x, lane = tid & 31;
   const u32 wmask = static_cast<u32>(W - 1);
@@ -202,11 +202,13 @@ __global__ void __launch_bounds__(BT, 1) k6_accumulate(
   if (tid == 0) {
     for (int s = 0; s < stages; ++s) mbar_init(&full_bar[s], 1);
     s_abort = 0;
-    s_dense_n = 0;
+    s_dense_n[0] = 0;
+    s_dense_n[1] = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   __syncthreads();
   u32 phase_bits = 0;  // bit s = parity to wait for on stage s
+  int dpar = 0;        // which dense-word counter the current chunk uses
 
   for (;;) {
     if (tid == 0) {
@@ -361,7 +363,7 @@ __global__ void __launch_bounds__(BT, 1) k6_accumulate(
               const u32 word = i == 0 ? word0 : bitmap[wb + i];
               const u32 wpc = __popc(word);
               if (wpc > 4) {
-                const int idx = atomicAdd(&s_dense_n, 1);
+                const int idx = atomicAdd(&s_dense_n[dpar], 1);
                 dense_list[idx] = static_cast<unsigned short>(wb + i);
                 word_prefix[wb + i] = ex;
               } else if (wpc) {
@@ -381,7 +383,7 @@ __global__ void __launch_bounds__(BT, 1) k6_accumulate(
             }
           }
           __syncthreads();
-          const int n_dense = s_dense_n;
+          const int n_dense = s_dense_n[dpar];
           constexpr int kWarps = BT / 32;
           for (int i = tid >> 5; i < n_dense; i += kWarps) {
             const int wi = dense_list[i];
@@ -398,8 +400,8 @@ __global__ void __launch_bounds__(BT, 1) k6_accumulate(
             __syncwarp();
             if (lane == 0) bitmap[wi] = 0u;
           }
-          __syncthreads();
-          if (tid == 0) s_dense_n = 0;
+          if (tid == 0) s_dense_n[dpar ^ 1] = 0;  // next chunk's counter: last read two barriers ago
+          dpar ^= 1;
         }
         __syncthreads();
         ++kw;
