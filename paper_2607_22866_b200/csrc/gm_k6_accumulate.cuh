@@ -118,6 +118,10 @@ __device__ __forceinline__ void acc_add(bool valid, u32 cl, V v, V* acc, u32* bi
 // result over the chunk's start in the staging buffer.  This is the paper's separate branch for light chunks
 // (Section III-A), with a sort where the paper uses a hash table.
 constexpr int kAccSmallChunk = 32;
+#ifndef GM_ACC_LIST_MIN
+#define GM_ACC_LIST_MIN 512
+#endif
+constexpr u32 kAccListMin = GM_ACC_LIST_MIN;  // chunks with more entries than this balance their dense words over the block
 
 template <typename V>
 __device__ __forceinline__ void small_chunk(int32_t* col, V* val, int n, int32_t* out_col, V* out_val,
@@ -172,15 +176,15 @@ __global__ void __launch_bounds__(BT, 1) k6_accumulate(
   constexpr int kAccTile = PT * BT;
   constexpr int kAccMetaCap = BT;
   const int n_words = W >> 5;
-  // layout: [ring cols][ring vals][acc][bitmap][meta base (i64)][meta off (i32)]
+  // layout: [ring cols][ring vals][acc][dense-word list][bitmap][chunk offsets of the metadata window]
   int32_t* r_col = reinterpret_cast<int32_t*>(smem_acc_raw);
   V* r_val = reinterpret_cast<V*>(smem_acc_raw + static_cast<size_t>(stages) * kAccTile * 4);
   unsigned char* after_ring = smem_acc_raw + static_cast<size_t>(stages) * kAccTile * (4 + (NUMERIC ? sizeof(V) : 0));
   V* acc = reinterpret_cast<V*>(after_ring);
-  u32* bitmap = reinterpret_cast<u32*>(after_ring + (NUMERIC ? static_cast<size_t>(W) * sizeof(V) : 0));
-  u32* word_prefix = bitmap + n_words;                                       // prefix of a dense word
-  unsigned short* dense_list = reinterpret_cast<unsigned short*>(word_prefix + n_words);  // n_words entries
-  int* m_off = reinterpret_cast<int*>(bitmap + 2 * n_words + ((n_words + 3) / 4) * 2);
+  // n_words entries {bits | word index, prefix}; W * sizeof(V) is a multiple of 128, so the list is 8-byte aligned
+  u64* dense_list = reinterpret_cast<u64*>(after_ring + (NUMERIC ? static_cast<size_t>(W) * sizeof(V) : 0));
+  u32* bitmap = reinterpret_cast<u32*>(dense_list + n_words);
+  int* m_off = reinterpret_cast<int*>(bitmap + n_words);
   __shared__ u64 full_bar[8];
   __shared__ u32 s_scan[33];
   __shared__ i64 s_seg[2];
@@ -192,6 +196,7 @@ __global__ void __launch_bounds__(BT, 1) k6_accumulate(
   constexpr u32 kStageBytesCol = kAccTile * 4;
   constexpr u32 kStageBytesVal = NUMERIC ? kAccTile * sizeof(V) : 0;
   constexpr int kPerThread = kAccTile / BT;  // elements of a full tile per thread
+  constexpr int kWarps = BT / 32;
   static_assert(kAccTile % BT == 0, "tile must be a multiple of the block");
   // the flush gives every thread wpt consecutive bitmap words (wpt is a power of two, at most 32)
   const int wpt = n_words > BT ? n_words / BT : 1;
@@ -339,6 +344,7 @@ __global__ void __launch_bounds__(BT, 1) k6_accumulate(
         // ---- chunk complete: flush
         __syncthreads();
         const int wb = tid * wpt;
+        const bool warp_has_words = (tid & ~31) * wpt < n_words;  // warp-uniform
         u32 pc = 0;
         u32 word0 = 0;  // the thread's first (for wpt == 1: only) word stays in a register
         if (wb < n_words) {
@@ -346,34 +352,49 @@ __global__ void __launch_bounds__(BT, 1) k6_accumulate(
           pc = __popc(word0);
           for (int i = 1; i < wpt; ++i) pc += __popc(bitmap[wb + i]);
         }
-        u32 total;
-        u32 ex = block_exclusive_scan(pc, s_scan, &total);
+        // Block-wide exclusive prefix with one barrier: every warp publishes its sum, then adds up the sums of
+        // the warps before it (and all of them, for the chunk's entry count) on its own.
+        const u32 inc = warp_inclusive_scan(pc);
+        if (lane == 31) s_scan[tid >> 5] = inc;
+        __syncthreads();
+        const u32 wsum = lane < kWarps ? s_scan[lane] : 0u;
+        const u32 total = __reduce_add_sync(0xffffffffu, wsum);
+        u32 ex = __reduce_add_sync(0xffffffffu, lane < (tid >> 5) ? wsum : 0u) + inc - pc;
         if (tid == 0) chunk_nnz[m0 + kw] = total;
         {
           // in place: the chunk's products [m_off[kw], ce) are all in shared memory or consumed by now
           int32_t* const c_col = x_col + lo_al + m_off[kw];
           V* const c_val = x_val + lo_al + m_off[kw];
-          constexpr i64 out0 = 0;
-          constexpr bool fits = true;
-          // Words with few bits are written by their owner.  Dense words cluster at the low end of the chunk
-          // (hub columns), i.e. in the first warps, so they go to a list that all warps then share out evenly;
-          // there the 32 lanes of a warp write one word at a time.
-          if (wb < n_words) {
+          // Words with few bits are written by their owner.  In a chunk with many entries the dense words
+          // cluster at the low end (hub columns), i.e. in the first warps, so they go to a list that all warps
+          // then share out evenly; there the 32 lanes of a warp write one word at a time.  A chunk with few
+          // entries cannot be far out of balance and skips the list and its barrier.
+          const bool use_list = total > kAccListMin;  // block-uniform
+          if (warp_has_words) {
             for (int i = 0; i < wpt; ++i) {
-              const u32 word = i == 0 ? word0 : bitmap[wb + i];
+              const u32 word = i == 0 ? word0 : (wb + i < n_words ? bitmap[wb + i] : 0u);
               const u32 wpc = __popc(word);
-              if (wpc > 4) {
-                const int idx = atomicAdd(&s_dense_n[dpar], 1);
-                dense_list[idx] = static_cast<unsigned short>(wb + i);
-                word_prefix[wb + i] = ex;
-              } else if (wpc) {
+              const bool dense = use_list && wpc > 4;
+              if (use_list) {
+                const u32 dmask = __ballot_sync(0xffffffffu, dense);
+                if (dmask) {
+                  int lbase = 0;
+                  if (lane == 0) lbase = atomicAdd(&s_dense_n[dpar], __popc(dmask));
+                  lbase = __shfl_sync(0xffffffffu, lbase, 0);
+                  if (dense)  // {bits, word index, prefix} in one entry: the write-out needs a single load
+                    dense_list[lbase + __popc(dmask & lanemask_lt())] =
+                        (static_cast<u64>((static_cast<u32>(wb + i) << 16) | ex) << 32) | word;
+                }
+              }
+              if (!dense && wpc) {
                 u32 wbits = word;
-                i64 p = out0 + ex;
+                u32 p = ex;
                 while (wbits) {
                   const int b = __ffs(wbits) - 1;
                   wbits &= wbits - 1;
                   const int slot = ((wb + i) << 5) + b;
-                  if (fits) { c_col[p] = static_cast<int32_t>(col_base + slot); c_val[p] = acc[slot]; }
+                  c_col[p] = static_cast<int32_t>(col_base + slot);
+                  c_val[p] = acc[slot];
                   acc[slot] = V(0);
                   ++p;
                 }
@@ -382,26 +403,32 @@ __global__ void __launch_bounds__(BT, 1) k6_accumulate(
               ex += wpc;
             }
           }
-          __syncthreads();
-          const int n_dense = s_dense_n[dpar];
-          constexpr int kWarps = BT / 32;
-          for (int i = tid >> 5; i < n_dense; i += kWarps) {
-            const int wi = dense_list[i];
-            const u32 word = bitmap[wi];
-            if ((word >> lane) & 1u) {
-              const int slot = (wi << 5) + lane;
-              if (fits) {
-                const i64 p = out0 + word_prefix[wi] + __popc(word & lanemask_lt());
+          if (use_list) {
+            __syncthreads();
+            const int n_dense = s_dense_n[dpar];
+            auto emit = [&](u64 e) {
+              const u32 word = static_cast<u32>(e);
+              const u32 hi32 = static_cast<u32>(e >> 32);
+              const int wi = static_cast<int>(hi32 >> 16);
+              if ((word >> lane) & 1u) {
+                const int slot = (wi << 5) + lane;
+                const u32 p = (hi32 & 0xffffu) + __popc(word & lanemask_lt());
                 c_col[p] = static_cast<int32_t>(col_base + slot);
                 c_val[p] = acc[slot];
+                acc[slot] = V(0);
               }
-              acc[slot] = V(0);
+              if (lane == 0) bitmap[wi] = 0u;
+            };
+            for (int i = tid >> 5; i < n_dense; i += 2 * kWarps) {  // two words in flight per warp
+              const u64 e0 = dense_list[i];
+              const bool two = i + kWarps < n_dense;
+              const u64 e1 = two ? dense_list[i + kWarps] : 0ull;
+              emit(e0);
+              if (two) emit(e1);
             }
-            __syncwarp();
-            if (lane == 0) bitmap[wi] = 0u;
+            if (tid == 0) s_dense_n[dpar ^ 1] = 0;  // next list's counter: last read two barriers ago
+            dpar ^= 1;
           }
-          if (tid == 0) s_dense_n[dpar ^ 1] = 0;  // next chunk's counter: last read two barriers ago
-          dpar ^= 1;
         }
         __syncthreads();
         ++kw;
