@@ -483,7 +483,17 @@ static int launch_accumulate(gm_plan* p, const Batch& b, const HeavyBatchState<V
   GM_CUDA(cudaMemsetAsync(p->ticket, 0, sizeof(int), st));
   GM_CUDA(cudaMemsetAsync(p->chunk_nnz, 0, static_cast<size_t>(hs.n_chunks) * sizeof(u32), st));
   const int per_sm = 1024 / bt;
-  static const int small_max = [] { const char* e = std::getenv("GM_SMALL_CHUNK"); return e ? std::atoi(e) : kAccSmallChunk; }();
+  // chunks of at most small_max products go to the warp-per-chunk kernel (GM_SMALL_CHUNK=0 sends all of them
+  // through the block-wide accumulator: a debugging aid)
+  static const int small_max = [] {
+    const char* e = std::getenv("GM_SMALL_CHUNK");
+    return e ? std::max(0, std::min(std::atoi(e), kAccSmallChunk)) : kAccSmallChunk;
+  }();
+  if (small_max > 0) {
+    k6_small_chunks<V><<<static_cast<unsigned>(p->num_sms * 16), kSmallWarps * 32, 0, st>>>(
+        hs.fin_col, hs.fin_val, hs.chunk_off, hs.n_chunks, W, small_max, p->chunk_nnz);
+    ++p->stats.launches;
+  }
   const unsigned grid = static_cast<unsigned>(std::min<i64>(n_segs, static_cast<i64>(p->num_sms) * per_sm));
 #define GM_ACC2(BT, PT)                                                                                              \
   do {                                                                                                               \

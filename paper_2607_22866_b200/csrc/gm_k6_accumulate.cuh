@@ -109,59 +109,163 @@ __device__ __forceinline__ void acc_add(bool valid, u32 cl, V v, V* acc, u32* bi
   }
 }
 
-// Small chunks.  Going through the block-wide accumulator costs every chunk a few microseconds of barriers
-// and prefix sums whatever it holds, and most chunks of a power-law product hold few products.  A chunk of at
-// most kAccSmallChunk products that lies completely inside the current tile is instead handled by ONE warp,
-// with no block-wide step at all, so that 32 such chunks are in progress per block: the warp sorts the chunk's
-// (column, value) pairs in place in the shared-memory tile (bitonic network with ascending-only comparators,
-// so a length that is not a power of two needs no padding), adds up runs of equal columns and writes the
-// result over the chunk's start in the staging buffer.  This is the paper's separate branch for light chunks
-// (Section III-A), with a sort where the paper uses a hash table.
-constexpr int kAccSmallChunk = 32;
+// Small chunks.  Going through the block-wide accumulator costs every chunk a few thousand cycles of barriers,
+// prefix sums and dependent shared-memory round trips whatever it holds, and most chunks of a power-law product
+// hold few products.  Chunks of at most kAccSmallChunk products are therefore handled before the streaming
+// kernel runs, by ONE warp each and with no block-wide step, so that every SM works on dozens of them at a
+// time: the warp loads the chunk, sorts (column, position) keys packed into one word in registers (bitonic
+// network of ascending-only comparators: one shuffle and one min/max per key and step), adds up runs of equal
+// columns in the original order and writes the result over the chunk's start in the staging buffer.  This
+// is the paper's separate branch for light chunks (Section III-A), with a sort where the paper uses a hash
+// table.  The streaming kernel skips these chunks.
+#ifndef GM_SMALL_PER_LANE
+#define GM_SMALL_PER_LANE 16
+#endif
+constexpr int kSmallMaxPerLane = GM_SMALL_PER_LANE;
+constexpr int kAccSmallChunk = 32 * kSmallMaxPerLane;
+constexpr int kSmallIdxBits = kSmallMaxPerLane == 32 ? 10 : (kSmallMaxPerLane == 16 ? 9 : 8);  // position of a product inside its chunk
+constexpr int kSmallWarps = 4;            // warps per block of the small-chunk kernel
 #ifndef GM_ACC_LIST_MIN
 #define GM_ACC_LIST_MIN 512
 #endif
 constexpr u32 kAccListMin = GM_ACC_LIST_MIN;  // chunks with more entries than this balance their dense words over the block
 
-template <typename V>
-__device__ __forceinline__ void small_chunk(int32_t* col, V* val, int n, int32_t* out_col, V* out_val,
-                                            u32* nnz_out) {
-  const int lane = threadIdx.x & 31;
-  int N = 1;
-  while (N < n) N <<= 1;
-  for (int k = 2; k <= N; k <<= 1) {
-    for (int j = k - 1, first = 1; j > 0; j = first ? (k >> 2) : (j >> 1), first = 0) {
-      for (int i = lane; i < n; i += 32) {
-        const int l = i ^ j;
-        if (l > i && l < n) {
-          const int32_t a = col[i], b = col[l];
-          if (a > b) {
-            col[i] = b; col[l] = a;
-            const V t = val[i]; val[i] = val[l]; val[l] = t;
-          }
+// Sorts 32 * K packed keys, K per lane, element e = r * 32 + lane in key[r]; ascending in e afterwards.
+template <int K>
+__device__ __forceinline__ void warp_sort_keys(u32 (&key)[K], int lane) {
+#pragma unroll
+  for (int k = 2; k <= 32 * K; k <<= 1) {
+    // first step of a merge: partner e ^ (k - 1); the lower position keeps the smaller key
+    if (k <= 32) {
+      const bool lower = (lane & (k >> 1)) == 0;
+#pragma unroll
+      for (int r = 0; r < K; ++r) {
+        const u32 o = __shfl_xor_sync(0xffffffffu, key[r], k - 1);
+        key[r] = lower ? min(key[r], o) : max(key[r], o);
+      }
+    } else {
+      const int rm = k / 32 - 1;  // partner register r ^ rm, partner lane lane ^ 31
+#pragma unroll
+      for (int r = 0; r < K; ++r) {
+        if ((r ^ rm) > r) {
+          const u32 a = key[r], b = key[r ^ rm];
+          const u32 oa = __shfl_xor_sync(0xffffffffu, b, 31);
+          const u32 ob = __shfl_xor_sync(0xffffffffu, a, 31);
+          key[r] = min(a, oa);
+          key[r ^ rm] = max(b, ob);
         }
       }
-      __syncwarp();
-      if (first && k == 2) break;  // k = 2 has only the mirror step
+    }
+    // the remaining steps: partner e ^ j for j = k/4, k/8, ..., 1
+#pragma unroll
+    for (int j = k >> 2; j > 0; j >>= 1) {
+      if (j >= 32) {
+        const int rj = j / 32;
+#pragma unroll
+        for (int r = 0; r < K; ++r) {
+          if ((r & rj) == 0) {
+            const u32 a = key[r], b = key[r | rj];
+            key[r] = min(a, b);
+            key[r | rj] = max(a, b);
+          }
+        }
+      } else {
+        const bool lower = (lane & j) == 0;
+#pragma unroll
+        for (int r = 0; r < K; ++r) {
+          const u32 o = __shfl_xor_sync(0xffffffffu, key[r], j);
+          key[r] = lower ? min(key[r], o) : max(key[r], o);
+        }
+      }
     }
   }
+}
+
+// One small chunk by one warp.  s_key / s_val: 32 * K entries of this warp's shared memory.
+template <typename V, int K>
+__device__ __forceinline__ void small_chunk(int32_t* col, V* val, int n, u32 wmask, u32* s_key, V* s_val,
+                                            u32* nnz_out) {
+  const int lane = threadIdx.x & 31;
+  u32 key[K];
+  int32_t c_first = 0;
+#pragma unroll
+  for (int r = 0; r < K; ++r) {
+    const int e = r * 32 + lane;
+    key[r] = 0xffffffffu;  // padding sorts to the end
+    if (e < n) {
+      const int32_t c = col[e];
+      if (e == 0) c_first = c;
+      key[r] = ((static_cast<u32>(c) & wmask) << kSmallIdxBits) | static_cast<u32>(e);
+      s_val[e] = val[e];
+    }
+  }
+  const u32 col_base = static_cast<u32>(__shfl_sync(0xffffffffu, c_first, 0)) & ~wmask;
+  warp_sort_keys<K>(key, lane);
+#pragma unroll
+  for (int r = 0; r < K; ++r) s_key[r * 32 + lane] = key[r];
+  __syncwarp();
   // runs of equal columns: the lane that owns a run's first element adds the run up and writes it
   int base = 0;
-  for (int b0 = 0; b0 < n; b0 += 32) {
-    const int i = b0 + lane;
-    const bool head = i < n && (i == 0 || col[i] != col[i - 1]);
-    const u32 heads = __ballot_sync(0xffffffffu, head);
-    if (head) {
-      const int32_t c = col[i];
-      V sum = val[i];
-      for (int q = i + 1; q < n && col[q] == c; ++q) sum += val[q];
-      const int p = base + __popc(heads & lanemask_lt());
-      out_col[p] = c;
-      out_val[p] = sum;
+#pragma unroll
+  for (int r = 0; r < K; ++r) {
+    if (r * 32 < n) {  // warp-uniform
+      const int e = r * 32 + lane;
+      const u32 c = key[r] >> kSmallIdxBits;
+      const bool head = e < n && (e == 0 || (s_key[e - 1] >> kSmallIdxBits) != c);
+      const u32 heads = __ballot_sync(0xffffffffu, head);
+      if (head) {
+        V sum = s_val[key[r] & ((1u << kSmallIdxBits) - 1u)];
+        for (int q = e + 1; q < n; ++q) {
+          const u32 kq = s_key[q];
+          if ((kq >> kSmallIdxBits) != c) break;
+          sum += s_val[kq & ((1u << kSmallIdxBits) - 1u)];
+        }
+        const int p = base + __popc(heads & lanemask_lt());
+        col[p] = static_cast<int32_t>(col_base | c);
+        val[p] = sum;
+      }
+      base += __popc(heads);
     }
-    base += __popc(heads);
   }
   if (lane == 0) *nnz_out = static_cast<u32>(base);
+  __syncwarp();  // the warp's shared memory is reused by its next chunk
+}
+
+template <typename V>
+__global__ void __launch_bounds__(kSmallWarps * 32) k6_small_chunks(
+    int32_t* x_col, V* x_val, const i64* __restrict__ chunk_off, i64 n_chunks, int W, int small_max,
+    u32* __restrict__ chunk_nnz) {
+  __shared__ u32 s_key[kSmallWarps][32 * kSmallMaxPerLane];
+  __shared__ V s_val[kSmallWarps][32 * kSmallMaxPerLane];
+  const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+  const u32 wmask = static_cast<u32>(W - 1);
+  const i64 n_groups = (n_chunks + 31) >> 5;
+  // a warp looks at 32 consecutive chunks at a time and works through the small ones among them
+  for (i64 g = static_cast<i64>(blockIdx.x) * kSmallWarps + w; g < n_groups; g += static_cast<i64>(gridDim.x) * kSmallWarps) {
+    const i64 k = (g << 5) + lane;
+    i64 cs = 0;
+    int cn = 0;
+    if (k < n_chunks) {
+      cs = chunk_off[k];
+      cn = static_cast<int>(min(chunk_off[k + 1] - cs, static_cast<i64>(INT_MAX)));
+    }
+    u32 todo = __ballot_sync(0xffffffffu, cn > 0 && cn <= small_max);
+    while (todo) {
+      const int src = __ffs(todo) - 1;
+      todo &= todo - 1;
+      const i64 s0 = __shfl_sync(0xffffffffu, cs, src);
+      const int n = __shfl_sync(0xffffffffu, cn, src);
+      int32_t* col = x_col + s0;
+      V* val = x_val + s0;
+      u32* out = &chunk_nnz[(g << 5) + src];
+      if (n <= 32) small_chunk<V, 1>(col, val, n, wmask, s_key[w], s_val[w], out);
+      else if (n <= 64) small_chunk<V, 2>(col, val, n, wmask, s_key[w], s_val[w], out);
+      else if (n <= 128) small_chunk<V, 4>(col, val, n, wmask, s_key[w], s_val[w], out);
+      else if (kSmallMaxPerLane == 8 || n <= 256) small_chunk<V, 8>(col, val, n, wmask, s_key[w], s_val[w], out);
+      else if (kSmallMaxPerLane == 16 || n <= 512) small_chunk<V, (kSmallMaxPerLane >= 16 ? 16 : 8)>(col, val, n, wmask, s_key[w], s_val[w], out);
+      else small_chunk<V, kSmallMaxPerLane>(col, val, n, wmask, s_key[w], s_val[w], out);
+    }
+  }
 }
 
 template <typename V, bool NUMERIC, int BT, int PT>
@@ -287,31 +391,19 @@ __global__ void __launch_bounds__(BT, 1) k6_accumulate(
           __syncthreads();
         }
         const int ce = m_off[kw + 1];
-        if (ce - pos <= small_max && ce <= tile_hi && pos == m_off[kw]) {
-          // at the start of a small chunk: how many of the next 32 chunks are small and end inside this tile?  Every warp
-          // evaluates the same shared-memory metadata, so the answer is uniform without a barrier.
+        if (ce - m_off[kw] <= small_max) {
+          // an empty chunk, or a small one that the small-chunk kernel has dealt with: how many of the next 32
+          // chunks are like that?  Every warp evaluates the same shared-memory metadata, so the answer is
+          // uniform without a barrier.
           const i64 kc = m0 + kw + lane;
-          bool small = false;
-          if (kc < k_end) {
-            const int cs = m_off[kw + lane], cend = m_off[kw + lane + 1];
-            small = cend <= tile_hi && cend - cs <= small_max;
-          }
-          const u32 not_small = ~__ballot_sync(0xffffffffu, small);
-          const int run = not_small ? __ffs(not_small) - 1 : 32;
-          if (run > 0) {
-            if (!s_abort) {
-              for (int w = tid >> 5; w < run; w += BT / 32) {  // one chunk per warp, round-robin
-                const int cs = m_off[kw + w], cn = m_off[kw + w + 1] - cs;
-                if (cn > 0) small_chunk<V>(tc + cs, tv + cs, cn, x_col + lo_al + cs, x_val + lo_al + cs, &chunk_nnz[m0 + kw + w]);
-              }
-            }
-            kw += run;
-            crow = (crow + static_cast<u32>(run)) & crow_mask;
-            pos = m_off[kw];
-            continue;
-          }
+          const bool skip = kc < k_end && m_off[kw + lane + 1] - m_off[kw + lane] <= small_max;
+          const u32 not_skip = ~__ballot_sync(0xffffffffu, skip);
+          const int run = not_skip ? __ffs(not_skip) - 1 : 32;  // >= 1
+          kw += run;
+          crow = (crow + static_cast<u32>(run)) & crow_mask;
+          pos = m_off[kw];
+          continue;
         }
-        if (ce <= pos) { ++kw; crow = (crow + 1u) & crow_mask; continue; }  // empty chunk
         const int sub_hi = min(tile_hi, ce);
         const u32 col_base = crow << log2W;
         if (!s_abort) {
@@ -398,8 +490,8 @@ __global__ void __launch_bounds__(BT, 1) k6_accumulate(
                   acc[slot] = V(0);
                   ++p;
                 }
-                bitmap[wb + i] = 0u;
               }
+              if (wpc) bitmap[wb + i] = 0u;  // a listed word's bits travel in its list entry
               ex += wpc;
             }
           }
@@ -408,23 +500,21 @@ __global__ void __launch_bounds__(BT, 1) k6_accumulate(
             const int n_dense = s_dense_n[dpar];
             auto emit = [&](u64 e) {
               const u32 word = static_cast<u32>(e);
-              const u32 hi32 = static_cast<u32>(e >> 32);
-              const int wi = static_cast<int>(hi32 >> 16);
               if ((word >> lane) & 1u) {
-                const int slot = (wi << 5) + lane;
+                const u32 hi32 = static_cast<u32>(e >> 32);
+                const int slot = static_cast<int>((hi32 >> 16) << 5) + lane;
                 const u32 p = (hi32 & 0xffffu) + __popc(word & lanemask_lt());
                 c_col[p] = static_cast<int32_t>(col_base + slot);
                 c_val[p] = acc[slot];
                 acc[slot] = V(0);
               }
-              if (lane == 0) bitmap[wi] = 0u;
             };
             for (int i = tid >> 5; i < n_dense; i += 2 * kWarps) {  // two words in flight per warp
               const u64 e0 = dense_list[i];
               const bool two = i + kWarps < n_dense;
               const u64 e1 = two ? dense_list[i + kWarps] : 0ull;
               emit(e0);
-              if (two) emit(e1);
+              emit(e1);
             }
             if (tid == 0) s_dense_n[dpar ^ 1] = 0;  // next list's counter: last read two barriers ago
             dpar ^= 1;
