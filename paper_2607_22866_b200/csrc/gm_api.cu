@@ -399,7 +399,8 @@ static int launch_light_one(gm_plan* p, const int32_t* rows, const int* n_rows_d
   constexpr int kGroups = BT / G;
   const size_t smem = kGroups * light_group_bytes<V, NUMERIC>(slots, cap);
   auto kern = k3_light_rows<V, G, LPN, BT, NUMERIC>;
-  if (smem > 48 * 1024) GM_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)));
+  // (static shared memory counts towards the 48 KB that need no opt-in)
+  if (smem > 32 * 1024) GM_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)));
   const unsigned grid = grid_for(n_rows_upper, kGroups, p->num_sms, 2048 / BT * 4);
   kern<<<grid, BT, smem, st>>>(p->A.row_ptr, p->A.col_idx, static_cast<const V*>(p->A.vals), p->B.row_ptr, p->B.col_idx,
                                static_cast<const V*>(p->B.vals), rows, n_rows_dev, slots, cap, p->row_nnz, c_row_ptr, c_col,
@@ -498,7 +499,7 @@ static int launch_accumulate(gm_plan* p, const Batch& b, const HeavyBatchState<V
 #define GM_ACC2(BT, PT)                                                                                              \
   do {                                                                                                               \
     auto kern = k6_accumulate<V, true, BT, PT>;                                                                      \
-    if (smem > 48 * 1024)                                                                                            \
+    if (smem > 32 * 1024)                                                                                            \
       GM_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)));     \
     kern<<<grid, BT, smem, st>>>(hs.fin_col, hs.fin_val, hs.chunk_off, hs.n_chunks, p->seg_first, n_segs, p->ticket, \
                                  hs.log2_cpr, W, stages, small_max, p->chunk_nnz, p->err);                                      \

@@ -124,11 +124,25 @@ __global__ void __launch_bounds__(BT) k3_light_rows(
     group_sync<G>();
     const i64 out0 = c_row_ptr[row];
     const int n = static_cast<int>(c_row_ptr[row + 1] - out0);
-    for (int s = t; s < slots; s += G) {
-      const int32_t c = keys[s];
-      if (c != kEmptyKey) {
-        const int idx = atomicAdd(&s_count[gid], 1);
-        if (idx < cap) sortbuf[idx] = (static_cast<u64>(static_cast<u32>(c)) << 32) | static_cast<u32>(s);
+    if constexpr (G >= 32) {
+      // one counter update per warp and step: the occupied lanes take consecutive places
+      const u32 lane = threadIdx.x & 31;
+      for (int s0 = 0; s0 < slots; s0 += G) {
+        const int s = s0 + t;
+        const int32_t c = s < slots ? keys[s] : kEmptyKey;
+        const u32 occ = __ballot_sync(0xffffffffu, c != kEmptyKey);
+        int idx = 0;
+        if (lane == 0 && occ) idx = atomicAdd(&s_count[gid], __popc(occ));
+        idx = __shfl_sync(0xffffffffu, idx, 0) + __popc(occ & lanemask_lt());
+        if (c != kEmptyKey && idx < cap) sortbuf[idx] = (static_cast<u64>(static_cast<u32>(c)) << 32) | static_cast<u32>(s);
+      }
+    } else {
+      for (int s = t; s < slots; s += G) {
+        const int32_t c = keys[s];
+        if (c != kEmptyKey) {
+          const int idx = atomicAdd(&s_count[gid], 1);
+          if (idx < cap) sortbuf[idx] = (static_cast<u64>(static_cast<u32>(c)) << 32) | static_cast<u32>(s);
+        }
       }
     }
     int n2 = 1;

@@ -53,17 +53,8 @@ int planner_params(int64_t c_cols, int dtype, size_t smem_bytes, const gm_plan_o
   // with cap * 8 + 1.5 * cap * se <= S, and as many slots as fit, at most alpha * cap.
   int64_t cap = 16;
   while ((cap * 2) * 8 + 3 * (cap * 2) * se / 2 <= S - reserve) cap *= 2;
-  // The capacity is an upper limit; the sort that follows accumulation costs n log^2 n, and on B200 rows above
-  // 4096 products measured cheaper on the heavy path than in a one-block-per-SM hash + sort.
-  int64_t tau = std::min<int64_t>(cap, 4096);
   if (o.tau < 0) return GM_ERR_INVALID_ARG;
-  if (o.tau > 0) {
-    if (o.tau > cap) return GM_ERR_INVALID_ARG;  // would not fit the light-row accumulator
-    tau = o.tau;
-  }
-  const int64_t top_cap = static_cast<int64_t>(pow2_ceil(static_cast<uint64_t>(std::max<int64_t>(tau, 16))));
-  out->tau = tau;
-  out->light_slots = static_cast<int32_t>(std::min<int64_t>(2 * top_cap, (S - reserve - 8 * top_cap) / se));
+  if (o.tau > cap) return GM_ERR_INVALID_ARG;  // would not fit the light-row accumulator
 
   // --- W = n_denseNumeric: columns one dense accumulator (values + bitmap) covers, power of two.
   int ctas = o.acc_ctas_per_sm ? o.acc_ctas_per_sm : 1;
@@ -92,6 +83,16 @@ int planner_params(int64_t c_cols, int dtype, size_t smem_bytes, const gm_plan_o
   const int64_t required = static_cast<int64_t>(pow2_ceil(static_cast<uint64_t>(need)));
   if (required > (int64_t{1} << 30)) return GM_ERR_CAPACITY;
   out->chunks_required = static_cast<int32_t>(required);
+
+  // --- default tau.  The capacity is an upper limit.  A light row pays for a hash table and an n log^2 n sort
+  // in one block; a heavy row pays per chunk (a one-warp register sort for the small ones).  Measured on
+  // B200: with up to 32 chunks per row the heavy path is cheaper from about 512 products on, with more
+  // chunks per row from about 1024 (R-MAT 20: 445 ms at 4096, 414 ms at 512; R-MAT 21 in fp64, 128 chunks:
+  // 610 ms at 4096, 530 ms at 1024).
+  int64_t tau = o.tau > 0 ? o.tau : std::min<int64_t>(cap, required <= 32 ? 512 : 1024);
+  const int64_t top_cap = static_cast<int64_t>(pow2_ceil(static_cast<uint64_t>(std::max<int64_t>(tau, 16))));
+  out->tau = tau;
+  out->light_slots = static_cast<int32_t>(std::min<int64_t>(2 * top_cap, (S - reserve - 8 * top_cap) / se));
 
   // --- n_chunksMax (Eq. 6) with n_groupRows = 2, 32 subgroups per work group, 4-byte histogram
   // counters and 8-byte offsets, half of s_LM given to the permuted elements; floored to a power

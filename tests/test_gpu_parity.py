@@ -277,3 +277,31 @@ def test_accumulators_per_sm_with_many_tiny_chunks(ctas):
     A, B, _ = gen.config_inputs(4, shrink=4)
     C, info, stats = check_product(A, B, acc_ctas_per_sm=ctas, tau=256)
     assert info.rows_heavy > 100 and info.params.acc_ctas_per_sm == ctas
+
+
+@pytest.mark.parametrize("dtype", [np.float32, np.float64])
+def test_chunk_sizes_around_the_warp_sort_widths(dtype):
+    # Chunks of 1 ... 600 products, with repeated columns, on both sides of every width of the one-warp sort
+    # (32, 64, 128, 256, 512 products) and of the hand-over to the block-wide accumulator.  Row r of B holds
+    # 2^r entries in chunk 1 (columns 1024..2047, drawn from 300 columns so that rows overlap) and one entry
+    # in chunk 0; a row of A picks the rows of B that spell its target size in binary.
+    rng = np.random.default_rng(17)
+    pool = 1024 + rng.choice(1024, 300, replace=False)
+    patB = np.zeros((10, 4096), bool)
+    for r in range(10):
+        patB[r, rng.choice(pool, min(1 << r, 300), replace=False)] = True
+        patB[r, r] = True
+    sizes_of_b = patB[:, 1024:2048].sum(axis=1)
+    B = csr_from_pattern(patB, rng.uniform(-1, 1, patB.shape), dtype)
+    targets = [1, 2, 31, 32, 33, 63, 64, 65, 127, 128, 129, 255, 256, 257, 300, 511]
+    patA = np.zeros((len(targets) + 3, 10), bool)
+    for i, n in enumerate(targets):
+        patA[i] = [(n >> r) & 1 for r in range(10)]
+    patA[len(targets)] = True                     # all rows: the largest chunk
+    patA[len(targets) + 1, [8, 9]] = True
+    patA[len(targets) + 2, [9]] = True
+    A = csr_from_pattern(patA, rng.uniform(-1, 1, patA.shape), dtype)
+    chunk1 = patA.astype(np.int64) @ sizes_of_b
+    assert chunk1.min() == 1 and (chunk1 > 512).any() and {32, 33, 256, 257}.issubset(set(chunk1.tolist()))
+    C, info, stats = check_product(A, B, tau=1, chunk_width=1024, max_fanout=4)
+    assert info.rows_heavy == int((chunk1 + patA.sum(axis=1) > 1).sum())

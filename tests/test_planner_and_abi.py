@@ -96,10 +96,10 @@ def test_b200_defaults():
         assert p.max_fanout == min(256, 1 << (raw.bit_length() - 1))
     assert p32.levels() == [32] and p64.levels() == [128]
     # light-row capacity: table (<= 2 slots per entry) + 64-bit sort buffer must fit s_LM; the default
-    # threshold stops at 4096 products (beyond that the sort costs more than the heavy path), the
-    # capacity itself is 8192 and can be asked for, 16384 cannot
+    # threshold is far below it (512 products with up to 32 chunks per row, 1024 with more: beyond that the
+    # sort costs more than the heavy path), the capacity itself is 8192 and can be asked for, 16384 cannot
+    assert (p32.tau, p32.light_slots) == (512, 1024) and (p64.tau, p64.light_slots) == (1024, 2048)
     for sv, p in ((4, p32), (8, p64)):
-        assert p.tau == 4096 and p.light_slots == 8192
         dt = np.float32 if sv == 4 else np.float64
         o = gm.PlanOpts(); o.tau = 8192
         q = gm.planner_params(1 << 20, dt, s, o)
