@@ -491,7 +491,7 @@ static int launch_accumulate(gm_plan* p, const Batch& b, const HeavyBatchState<V
     return e ? std::max(0, std::min(std::atoi(e), kAccSmallChunk)) : kAccSmallChunk;
   }();
   if (small_max > 0) {
-    k6_small_chunks<V><<<static_cast<unsigned>(p->num_sms * 16), kSmallWarps * 32, 0, st>>>(
+    k6_small_chunks<V><<<static_cast<unsigned>(p->num_sms * 8), kSmallWarps * 32, 0, st>>>(
         hs.fin_col, hs.fin_val, hs.chunk_off, hs.n_chunks, W, small_max, p->chunk_nnz);
     ++p->stats.launches;
   }

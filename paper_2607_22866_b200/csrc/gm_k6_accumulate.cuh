@@ -131,53 +131,53 @@ constexpr int kSmallWarps = 4;            // warps per block of the small-chunk 
 constexpr u32 kAccListMin = GM_ACC_LIST_MIN;  // chunks with more entries than this balance their dense words over the block
 
 // Sorts 32 * K packed keys, K per lane, element e = r * 32 + lane in key[r]; ascending in e afterwards.
+// Steps whose partner sits in another lane are the same instruction sequence for every step width, so they run
+// as loops over the width; only the steps that pair registers are unrolled.  (Fully unrolled, the networks of
+// all K together did not fit the instruction cache, and the warps of a block run different K.)
 template <int K>
 __device__ __forceinline__ void warp_sort_keys(u32 (&key)[K], int lane) {
+  auto lane_step = [&](int mask, bool lower) {  // partner: same register, lane ^ mask; the lower lane keeps the smaller key
 #pragma unroll
-  for (int k = 2; k <= 32 * K; k <<= 1) {
-    // first step of a merge: partner e ^ (k - 1); the lower position keeps the smaller key
-    if (k <= 32) {
-      const bool lower = (lane & (k >> 1)) == 0;
+    for (int r = 0; r < K; ++r) {
+      const u32 o = __shfl_xor_sync(0xffffffffu, key[r], mask);
+      key[r] = lower ? min(key[r], o) : max(key[r], o);
+    }
+  };
+  // merges inside one register row (k = 2 .. 32): first step partner e ^ (k - 1), then e ^ j for j = k/4 .. 1
+#pragma unroll 1
+  for (int k = 2; k <= 32; k <<= 1) {
+    lane_step(k - 1, (lane & (k >> 1)) == 0);
+#pragma unroll 1
+    for (int j = k >> 2; j > 0; j >>= 1) lane_step(j, (lane & j) == 0);
+  }
+  // merges across register rows (k = 64 .. 32 K)
 #pragma unroll
-      for (int r = 0; r < K; ++r) {
-        const u32 o = __shfl_xor_sync(0xffffffffu, key[r], k - 1);
-        key[r] = lower ? min(key[r], o) : max(key[r], o);
+  for (int k = 64; k <= 32 * K; k <<= 1) {
+    const int rm = k / 32 - 1;  // first step: partner register r ^ rm, partner lane lane ^ 31
+#pragma unroll
+    for (int r = 0; r < K; ++r) {
+      if ((r ^ rm) > r) {
+        const u32 a = key[r], b = key[r ^ rm];
+        const u32 oa = __shfl_xor_sync(0xffffffffu, b, 31);
+        const u32 ob = __shfl_xor_sync(0xffffffffu, a, 31);
+        key[r] = min(a, oa);
+        key[r ^ rm] = max(b, ob);
       }
-    } else {
-      const int rm = k / 32 - 1;  // partner register r ^ rm, partner lane lane ^ 31
+    }
+#pragma unroll
+    for (int j = k >> 2; j >= 32; j >>= 1) {  // partner in the same lane
+      const int rj = j / 32;
 #pragma unroll
       for (int r = 0; r < K; ++r) {
-        if ((r ^ rm) > r) {
-          const u32 a = key[r], b = key[r ^ rm];
-          const u32 oa = __shfl_xor_sync(0xffffffffu, b, 31);
-          const u32 ob = __shfl_xor_sync(0xffffffffu, a, 31);
-          key[r] = min(a, oa);
-          key[r ^ rm] = max(b, ob);
+        if ((r & rj) == 0) {
+          const u32 a = key[r], b = key[r | rj];
+          key[r] = min(a, b);
+          key[r | rj] = max(a, b);
         }
       }
     }
-    // the remaining steps: partner e ^ j for j = k/4, k/8, ..., 1
-#pragma unroll
-    for (int j = k >> 2; j > 0; j >>= 1) {
-      if (j >= 32) {
-        const int rj = j / 32;
-#pragma unroll
-        for (int r = 0; r < K; ++r) {
-          if ((r & rj) == 0) {
-            const u32 a = key[r], b = key[r | rj];
-            key[r] = min(a, b);
-            key[r | rj] = max(a, b);
-          }
-        }
-      } else {
-        const bool lower = (lane & j) == 0;
-#pragma unroll
-        for (int r = 0; r < K; ++r) {
-          const u32 o = __shfl_xor_sync(0xffffffffu, key[r], j);
-          key[r] = lower ? min(key[r], o) : max(key[r], o);
-        }
-      }
-    }
+#pragma unroll 1
+    for (int j = 16; j > 0; j >>= 1) lane_step(j, (lane & j) == 0);
   }
 }
 
