@@ -37,10 +37,10 @@ DEFAULT_CONFIG = 2  # R-MAT scale 20, edge factor 16, fp32: the largest fp32 pow
 
 
 # DRAM bytes per launch (ncu dram__bytes_read.sum + dram__bytes_write.sum) over the algorithmic bytes of the same
-# launch, measured on a scaled-down case of the same kernels (R-MAT scale 17, 134 M products per batch: see
+# launch, measured on a scaled-down case of the same kernels (R-MAT scale 17, 1.09 G products per step: see
 # profiles/dram_traffic_rmat17_f32.md).  Traffic grows in proportion to the products processed, so a full-size
 # launch is the algorithmic figure times this ratio.
-TRAFFIC_RATIO = {"k4_expand": 1.05, "k5b_multisplit": 1.03, "k6_accumulate": 1.00, "k7_gather": 1.08}
+TRAFFIC_RATIO = {"k4_expand": 1.03, "k5b_multisplit": 0.99, "k6_small_chunks": 0.73, "k6_accumulate": 1.01, "k7_gather": 0.99}
 
 
 def _peaks():
@@ -196,6 +196,7 @@ def kernel_table(info, stats_avg, sv, nnz_b, n_light_entries_a):
     L = p.n_levels
     nnz_c, nnz_ch = stats_avg["c_nnz"], stats_avg["c_nnz_heavy"]
     chunks = stats_avg["final_chunks"]
+    e_small, nnz_small = stats_avg["small_chunk_products"], stats_avg["small_chunk_entries"]
     parents = [rows_h]
     for l in range(L):
         parents.append(parents[-1] * p.fanout[l])
@@ -207,7 +208,9 @@ def kernel_table(info, stats_avg, sv, nnz_b, n_light_entries_a):
         "k4_expand": (se * e + se * nnz_b + 24 * info.nnz_a_heavy, stats_avg["ms_expand"]),
         "k5a_histogram": (hist, stats_avg["ms_histogram"]),
         "k5b_multisplit": (split, stats_avg["ms_multisplit"]),
-        "k6_accumulate": (se * e + se * nnz_ch + 12 * chunks, stats_avg["ms_accumulate"]),
+        # chunks of few products are sorted by one warp each; the streaming kernel owes the rest
+        "k6_small_chunks": (se * e_small + se * nnz_small + 12 * chunks, stats_avg["ms_small_chunks"]),
+        "k6_accumulate": (se * (e - e_small) + se * (nnz_ch - nnz_small) + 12 * chunks, stats_avg["ms_accumulate"]),
         "k7_gather": (2 * se * nnz_ch + 24 * chunks, stats_avg["ms_gather"]),
     }
     return {k: {"bytes": int(b), "ms": float(ms), "gbs": (b / ms / 1e6 if ms > 0 else 0.0)} for k, (b, ms) in tbl.items()}
@@ -336,7 +339,7 @@ def main():
     n_b = max(int(info.n_batches), 1)
     per_launch = {"k4_expand": n_b, "k5a_histogram": n_b * max(info.params.n_levels, 1),
                   "k5b_multisplit": n_b * max(info.params.n_levels, 1), "k6_accumulate": n_b,
-                  "k7_gather": n_b}.get(dom, 1)
+                  "k6_small_chunks": n_b, "k7_gather": n_b}.get(dom, 1)
     roofline = {"kernel": dom, "bound": "hbm", "achieved": kt[dom]["gbs"], "peak": peak, "unit": "GB/s",
                 "frac": kt[dom]["gbs"] / peak, "peak_kind": f"of {peak_kind}",
                 "traffic": (kt[dom]["bytes"] / per_launch * TRAFFIC_RATIO[dom]) if dom in TRAFFIC_RATIO else None,

@@ -117,9 +117,12 @@ typedef struct gm_exec_stats {
   int64_t staged_products;     /* products written to the staging buffer (all batches)         */
   int64_t final_chunks;        /* (row, chunk) pairs handed to the accumulate kernel           */
   int64_t launches;            /* kernels launched by this execute                             */
+  int64_t small_chunk_products; /* products in chunks handled by the one-warp-per-chunk kernel   */
+  int64_t small_chunk_entries;  /* entries of C those chunks produced                            */
   float ms_light_symbolic, ms_light_numeric, ms_expand, ms_histogram, ms_multisplit,
       ms_accumulate, ms_gather, ms_scan, ms_total;
-  float reserved[5];
+  float ms_small_chunks;       /* the one-warp-per-chunk kernel; ms_accumulate is the streaming kernel alone */
+  float reserved[4];
 } gm_exec_stats;
 
 typedef struct gm_plan gm_plan; /* opaque, owned by the library */

@@ -69,10 +69,11 @@ class PlanInfo(ctypes.Structure):
 class ExecStats(ctypes.Structure):
     _fields_ = [("c_nnz", ctypes.c_int64), ("c_nnz_heavy", ctypes.c_int64), ("c_capacity", ctypes.c_int64), ("staged_products", ctypes.c_int64),
                 ("final_chunks", ctypes.c_int64), ("launches", ctypes.c_int64),
+                ("small_chunk_products", ctypes.c_int64), ("small_chunk_entries", ctypes.c_int64),
                 ("ms_light_symbolic", ctypes.c_float), ("ms_light_numeric", ctypes.c_float),
                 ("ms_expand", ctypes.c_float), ("ms_histogram", ctypes.c_float), ("ms_multisplit", ctypes.c_float),
                 ("ms_accumulate", ctypes.c_float), ("ms_gather", ctypes.c_float), ("ms_scan", ctypes.c_float),
-                ("ms_total", ctypes.c_float), ("reserved", ctypes.c_float * 5)]
+                ("ms_total", ctypes.c_float), ("ms_small_chunks", ctypes.c_float), ("reserved", ctypes.c_float * 4)]
 
 
 _ALLOC_FN = ctypes.CFUNCTYPE(ctypes.c_void_p, ctypes.c_size_t, ctypes.c_void_p, ctypes.c_void_p)

@@ -92,7 +92,7 @@ struct Buf {
 // plan
 // ------------------------------------------------------------------------------------------------
 struct PhaseTimes {
-  enum Phase { kLightSym, kLightNum, kExpand, kHist, kSplit, kAccSym, kAccNum, kScan, kCount };
+  enum Phase { kLightSym, kLightNum, kExpand, kHist, kSplit, kAccSym, kAccNum, kAccSmall, kScan, kCount };
   struct Rec { int phase; cudaEvent_t a, b; };
   std::vector<Rec> recs;
   std::vector<cudaEvent_t> pool;
@@ -154,7 +154,7 @@ struct gm_plan {
   int* num_fill = nullptr;         // 8
   int32_t* row_nnz = nullptr;      // nA
   int64_t* scan_tmp = nullptr;
-  int64_t* c_total = nullptr;      // running nnz(C) (device carry)
+  int64_t* c_total = nullptr;      // [0] running nnz(C) (device carry), [1] heavy entries, [2] products and [3] entries of small chunks
   int* err = nullptr;
   // heavy workspace
   int32_t* stage_col[2]{};
@@ -264,7 +264,7 @@ static int build_plan(gm_plan* p, cudaStream_t st) {
   GM_TRY(plan_alloc(p, &heavy_pos, static_cast<size_t>(nA) + 1, st));
   GM_TRY(plan_alloc(p, &totals, 1, st));
   GM_TRY(plan_alloc(p, &p->row_nnz, static_cast<size_t>(nA) + 1, st));
-  GM_TRY(plan_alloc(p, &p->c_total, 2, st));
+  GM_TRY(plan_alloc(p, &p->c_total, 4, st));
   GM_TRY(plan_alloc(p, &p->scan_tmp, static_cast<size_t>(scan_tmp_elems(std::max<i64>(std::max(nnzA, nA), 1))), st));
   GM_CUDA(cudaMemsetAsync(totals, 0, sizeof(K1Totals), st));
   if (nnzA > 0) k1_nz_len<<<grid_for(nnzA, 256, p->num_sms, 32), 256, 0, st>>>(A.col_idx, nnzA, B.row_ptr, nz_len);
@@ -491,10 +491,14 @@ static int launch_accumulate(gm_plan* p, const Batch& b, const HeavyBatchState<V
     return e ? std::max(0, std::min(std::atoi(e), kAccSmallChunk)) : kAccSmallChunk;
   }();
   if (small_max > 0) {
+    p->times.begin(PhaseTimes::kAccSmall, st);
     k6_small_chunks<V><<<static_cast<unsigned>(p->num_sms * 8), kSmallWarps * 32, 0, st>>>(
-        hs.fin_col, hs.fin_val, hs.chunk_off, hs.n_chunks, W, small_max, p->chunk_nnz);
+        hs.fin_col, hs.fin_val, hs.chunk_off, hs.n_chunks, W, small_max, p->chunk_nnz,
+        reinterpret_cast<u64*>(p->c_total + 2));
     ++p->stats.launches;
+    p->times.end(st);
   }
+  p->times.begin(PhaseTimes::kAccNum, st);
   const unsigned grid = static_cast<unsigned>(std::min<i64>(n_segs, static_cast<i64>(p->num_sms) * per_sm));
 #define GM_ACC2(BT, PT)                                                                                              \
   do {                                                                                                               \
@@ -511,6 +515,7 @@ static int launch_accumulate(gm_plan* p, const Batch& b, const HeavyBatchState<V
   else GM_ACC(128);
 #undef GM_ACC
 #undef GM_ACC2
+  p->times.end(st);
   p->stats.launches += 2;
   GM_CUDA(cudaGetLastError());
   return GM_OK;
@@ -615,9 +620,7 @@ static int heavy_batch_front(gm_plan* p, const Batch& b, HeavyBatchState<V>* hs,
   p->stats.final_chunks += n_par;
   p->stats.staged_products += b.elems;
 
-  tm.begin(PhaseTimes::kAccNum, st);
-  GM_TRY((launch_accumulate<V>(p, b, *hs, st)));
-  tm.end(st);
+  GM_TRY((launch_accumulate<V>(p, b, *hs, st)));  // (records its own two phases)
   tm.begin(PhaseTimes::kScan, st);
   exclusive_scan<u32, i64>(p->chunk_nnz, p->chunk_nnz_off, hs->n_chunks, p->scan_tmp, nullptr, nullptr, nullptr, st);
   k_heavy_row_counts<<<grid_for(rows_b, 256, p->num_sms), 256, 0, st>>>(p->chunk_nnz_off, hs->log2_cpr, rows_b, p->x_heavy,
@@ -652,7 +655,7 @@ static int execute_t(gm_plan* p, cudaStream_t st, gm_csr* C) {
 
   GM_CUDA(cudaMemsetAsync(p->err, 0, sizeof(int), st));
   GM_CUDA(cudaMemsetAsync(p->row_nnz, 0, static_cast<size_t>(nA + 1) * sizeof(int32_t), st));
-  GM_CUDA(cudaMemsetAsync(p->c_total, 0, 2 * sizeof(int64_t), st));
+  GM_CUDA(cudaMemsetAsync(p->c_total, 0, 4 * sizeof(int64_t), st));
 
   // ---- result row_ptr
   i64* c_row_ptr = static_cast<i64*>(dev_alloc(static_cast<size_t>(nA + 1) * sizeof(i64), st));
@@ -770,7 +773,8 @@ static int execute_t(gm_plan* p, cudaStream_t st, gm_csr* C) {
     }
   }
   if (tm.enabled) cudaEventRecord(ev_total1, st);
-  cudaMemcpyAsync(&heavy_total, p->c_total + 1, sizeof(i64), cudaMemcpyDeviceToHost, st);
+  i64 tail_totals[3] = {0, 0, 0};  // heavy entries, small-chunk products, small-chunk entries
+  cudaMemcpyAsync(tail_totals, p->c_total + 1, 3 * sizeof(i64), cudaMemcpyDeviceToHost, st);
   cudaError_t e1 = cudaMemcpyAsync(&dev_err, p->err, sizeof(int), cudaMemcpyDeviceToHost, st);
   cudaError_t e2 = cudaStreamSynchronize(st);
   if (e1 != cudaSuccess || e2 != cudaSuccess) {
@@ -784,7 +788,10 @@ static int execute_t(gm_plan* p, cudaStream_t st, gm_csr* C) {
   }
 #undef GM_TRY_C
   p->stats.c_nnz = total;
+  heavy_total = tail_totals[0];
   p->stats.c_nnz_heavy = heavy_total;
+  p->stats.small_chunk_products = tail_totals[1];
+  p->stats.small_chunk_entries = tail_totals[2];
   p->stats.c_capacity = capacity;
   if (tm.enabled) {
     float ph[PhaseTimes::kCount];
@@ -796,6 +803,7 @@ static int execute_t(gm_plan* p, cudaStream_t st, gm_csr* C) {
     p->stats.ms_multisplit = ph[PhaseTimes::kSplit];
     p->stats.ms_gather = ph[PhaseTimes::kAccSym];
     p->stats.ms_accumulate = ph[PhaseTimes::kAccNum];
+    p->stats.ms_small_chunks = ph[PhaseTimes::kAccSmall];
     p->stats.ms_scan = ph[PhaseTimes::kScan];
     cudaEventElapsedTime(&p->stats.ms_total, ev_total0, ev_total1);
   }

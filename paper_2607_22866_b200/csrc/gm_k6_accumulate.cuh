@@ -183,8 +183,8 @@ __device__ __forceinline__ void warp_sort_keys(u32 (&key)[K], int lane) {
 
 // One small chunk by one warp.  s_key / s_val: 32 * K entries of this warp's shared memory.
 template <typename V, int K>
-__device__ __forceinline__ void small_chunk(int32_t* col, V* val, int n, u32 wmask, u32* s_key, V* s_val,
-                                            u32* nnz_out) {
+__device__ __forceinline__ int small_chunk(int32_t* col, V* val, int n, u32 wmask, u32* s_key, V* s_val,
+                                           u32* nnz_out) {
   const int lane = threadIdx.x & 31;
   u32 key[K];
   int32_t c_first = 0;
@@ -229,17 +229,20 @@ __device__ __forceinline__ void small_chunk(int32_t* col, V* val, int n, u32 wma
   }
   if (lane == 0) *nnz_out = static_cast<u32>(base);
   __syncwarp();  // the warp's shared memory is reused by its next chunk
+  return base;
 }
 
 template <typename V>
 __global__ void __launch_bounds__(kSmallWarps * 32) k6_small_chunks(
     int32_t* x_col, V* x_val, const i64* __restrict__ chunk_off, i64 n_chunks, int W, int small_max,
-    u32* __restrict__ chunk_nnz) {
+    u32* __restrict__ chunk_nnz,
+    u64* __restrict__ totals) {  // [0] += products, [1] += entries of the chunks handled here (statistics)
   __shared__ u32 s_key[kSmallWarps][32 * kSmallMaxPerLane];
   __shared__ V s_val[kSmallWarps][32 * kSmallMaxPerLane];
   const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
   const u32 wmask = static_cast<u32>(W - 1);
   const i64 n_groups = (n_chunks + 31) >> 5;
+  u64 sum_n = 0, sum_out = 0;
   // a warp looks at 32 consecutive chunks at a time and works through the small ones among them
   for (i64 g = static_cast<i64>(blockIdx.x) * kSmallWarps + w; g < n_groups; g += static_cast<i64>(gridDim.x) * kSmallWarps) {
     const i64 k = (g << 5) + lane;
@@ -258,13 +261,20 @@ __global__ void __launch_bounds__(kSmallWarps * 32) k6_small_chunks(
       int32_t* col = x_col + s0;
       V* val = x_val + s0;
       u32* out = &chunk_nnz[(g << 5) + src];
-      if (n <= 32) small_chunk<V, 1>(col, val, n, wmask, s_key[w], s_val[w], out);
-      else if (n <= 64) small_chunk<V, 2>(col, val, n, wmask, s_key[w], s_val[w], out);
-      else if (n <= 128) small_chunk<V, 4>(col, val, n, wmask, s_key[w], s_val[w], out);
-      else if (kSmallMaxPerLane == 8 || n <= 256) small_chunk<V, 8>(col, val, n, wmask, s_key[w], s_val[w], out);
-      else if (kSmallMaxPerLane == 16 || n <= 512) small_chunk<V, (kSmallMaxPerLane >= 16 ? 16 : 8)>(col, val, n, wmask, s_key[w], s_val[w], out);
-      else small_chunk<V, kSmallMaxPerLane>(col, val, n, wmask, s_key[w], s_val[w], out);
+      int m;
+      if (n <= 32) m = small_chunk<V, 1>(col, val, n, wmask, s_key[w], s_val[w], out);
+      else if (n <= 64) m = small_chunk<V, 2>(col, val, n, wmask, s_key[w], s_val[w], out);
+      else if (n <= 128) m = small_chunk<V, 4>(col, val, n, wmask, s_key[w], s_val[w], out);
+      else if (kSmallMaxPerLane == 8 || n <= 256) m = small_chunk<V, 8>(col, val, n, wmask, s_key[w], s_val[w], out);
+      else if (kSmallMaxPerLane == 16 || n <= 512) m = small_chunk<V, (kSmallMaxPerLane >= 16 ? 16 : 8)>(col, val, n, wmask, s_key[w], s_val[w], out);
+      else m = small_chunk<V, kSmallMaxPerLane>(col, val, n, wmask, s_key[w], s_val[w], out);
+      sum_n += static_cast<u64>(n);
+      sum_out += static_cast<u64>(m);
     }
+  }
+  if (lane == 0 && sum_n) {
+    atomicAdd(&totals[0], sum_n);
+    atomicAdd(&totals[1], sum_out);
   }
 }
 
