@@ -394,6 +394,17 @@ def e2e_leg(gm, torch, A, B, nnz, products, steps):
         h.row_ptr, h.col, h.val = pinned(M.row_ptr), pinned(M.col), pinned(M.val)
         return h
 
+    # C comes back into host buffers of nnz(C) entries: leave the leg out rather than have the host run out of memory
+    need = nnz * (4 + sv) + 2 * (A.nnz + (0 if B is A else B.nnz)) * (4 + sv)
+    try:
+        import psutil
+        avail = psutil.virtual_memory().available
+    except Exception:
+        avail = None
+    if avail is not None and need > 0.45 * avail:
+        return {"value": None, "unit": "GFLOP/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0,
+                "skipped": f"host buffers of {need / 1e9:.0f} GB for A, B and C do not fit beside the generator's "
+                           f"copies in {avail / 1e9:.0f} GB of available host memory"}
     hA = host_csr(A)
     hB = hA if B is A else host_csr(B)
     pin = True

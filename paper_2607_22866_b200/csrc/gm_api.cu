@@ -227,10 +227,12 @@ static int build_plan(gm_plan* p, cudaStream_t st) {
 
   int dev = 0;
   GM_CUDA(cudaGetDevice(&dev));
-  cudaDeviceProp prop;
-  GM_CUDA(cudaGetDeviceProperties(&prop, dev));
-  p->num_sms = prop.multiProcessorCount;
-  if (p->smem_bytes > prop.sharedMemPerBlockOptin)
+  // (two attribute queries: cudaGetDeviceProperties fills in the whole structure and takes milliseconds)
+  int num_sms = 0, smem_optin = 0;
+  GM_CUDA(cudaDeviceGetAttribute(&num_sms, cudaDevAttrMultiProcessorCount, dev));
+  GM_CUDA(cudaDeviceGetAttribute(&smem_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev));
+  p->num_sms = num_sms;
+  if (p->smem_bytes > static_cast<size_t>(smem_optin))
     return fail(GM_ERR_UNSUPPORTED_SMEM, "smem_bytes exceeds the device's opt-in shared memory per block");
   {
     const int rc = planner_params(B.n_cols, A.dtype, p->smem_bytes, &p->opts, &info.params);
