@@ -200,13 +200,18 @@ def kernel_table(info, stats_avg, sv, nnz_b, n_light_entries_a):
     parents = [rows_h]
     for l in range(L):
         parents.append(parents[-1] * p.fanout[l])
-    hist = sum(4 * e + 8 * (parents[l] + 1) + 4 * parents[l + 1] for l in range(L))
-    split = sum(2 * se * e + 8 * (parents[l] + 1) + 8 * parents[l + 1] for l in range(L))
+    # the expansion writes the first level's children itself (level0_direct): no pass over the staging buffer for
+    # that level, only per-segment run starts (read two child-boundary rows of B, write one row of prefixes)
+    l0 = 1 if (L > 0 and info.level0_direct) else 0
+    hist = sum(4 * e + 8 * (parents[l] + 1) + 4 * parents[l + 1] for l in range(l0, L))
+    split = sum(2 * se * e + 8 * (parents[l] + 1) + 8 * parents[l + 1] for l in range(l0, L))
+    seg_tables = (12 * p.fanout[0] * info.nnz_a_heavy + 4 * parents[1]) if l0 else 0
     tbl = {
         "k3_light_symbolic": (4 * n_light_entries_a + 8 * info.rows_light + 4 * nnz_b, stats_avg["ms_light_symbolic"]),
         "k3_light_numeric": (se * n_light_entries_a + se * nnz_b + se * (nnz_c - nnz_ch), stats_avg["ms_light_numeric"]),
-        "k4_expand": (se * e + se * nnz_b + 24 * info.nnz_a_heavy, stats_avg["ms_expand"]),
-        "k5a_histogram": (hist, stats_avg["ms_histogram"]),
+        "k4_expand": (se * e + se * nnz_b + 24 * info.nnz_a_heavy + (4 * p.fanout[0] * info.nnz_a_heavy if l0 else 0),
+                      stats_avg["ms_expand"]),
+        "k5a_histogram": (hist + seg_tables, stats_avg["ms_histogram"]),
         "k5b_multisplit": (split, stats_avg["ms_multisplit"]),
         # chunks of few products are sorted by one warp each; the streaming kernel owes the rest
         "k6_small_chunks": (se * e_small + se * nnz_small + 12 * chunks, stats_avg["ms_small_chunks"]),
@@ -337,8 +342,9 @@ def main():
     kt = kernel_table(info, stats_avg, sv, B.nnz, n_light_entries_a)
     dom = max(kt, key=lambda k: kt[k]["ms"])
     n_b = max(int(info.n_batches), 1)
-    per_launch = {"k4_expand": n_b, "k5a_histogram": n_b * max(info.params.n_levels, 1),
-                  "k5b_multisplit": n_b * max(info.params.n_levels, 1), "k6_accumulate": n_b,
+    n_split = max(info.params.n_levels - (1 if info.level0_direct else 0), 1)
+    per_launch = {"k4_expand": n_b, "k5a_histogram": n_b * n_split,
+                  "k5b_multisplit": n_b * n_split, "k6_accumulate": n_b,
                   "k6_small_chunks": n_b, "k7_gather": n_b}.get(dom, 1)
     roofline = {"kernel": dom, "bound": "hbm", "achieved": kt[dom]["gbs"], "peak": peak, "unit": "GB/s",
                 "frac": kt[dom]["gbs"] / peak, "peak_kind": f"of {peak_kind}",

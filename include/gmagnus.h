@@ -74,7 +74,11 @@ typedef struct gm_plan_opts {
   int32_t separate_histogram; /* 1: always run the stand-alone histogram kernel per level      */
   int32_t validate_inputs; /* 1: check row_ptr / col_idx of A and B on the device first        */
   int32_t single_stream;   /* 1: do not overlap the light and heavy paths on forked streams    */
-  int32_t reserved[7];
+  int32_t level0_multisplit; /* first multisplit level: 1 = separate histogram and multisplit passes over
+                              the staging buffer (Algorithm 5 as printed); 2 = the expansion kernel writes
+                              the first level's children itself; 0 (default) = the latter when the heavy
+                              rows' segments are long compared with the fan-out, else the former        */
+  int32_t reserved[6];
 } gm_plan_opts;
 
 /* What the host planner derives from (C.m, value size, smem_bytes): Section III-D. */
@@ -105,6 +109,7 @@ typedef struct gm_plan_info {
   int64_t workspace_bytes; /* device memory held by the plan                                   */
   int64_t light_bin_rows[8]; /* light rows per size class of the symbolic pass                 */
   int64_t launches;        /* kernels launched while planning                                  */
+  int64_t level0_direct;   /* 1: the expansion kernel writes the first level's children itself  */
 } gm_plan_info;
 
 /* Filled by the most recent gm_spgemm_execute on the plan.  Times are CUDA-event milliseconds on

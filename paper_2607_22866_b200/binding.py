@@ -43,7 +43,7 @@ class PlanOpts(ctypes.Structure):
                 ("acc_ctas_per_sm", ctypes.c_int32), ("stage_elems", ctypes.c_int64),
                 ("c_capacity", ctypes.c_int64), ("separate_histogram", ctypes.c_int32),
                 ("validate_inputs", ctypes.c_int32), ("single_stream", ctypes.c_int32),
-                ("reserved", ctypes.c_int32 * 7)]
+                ("level0_multisplit", ctypes.c_int32), ("reserved", ctypes.c_int32 * 6)]
 
 
 class Params(ctypes.Structure):
@@ -63,7 +63,7 @@ class PlanInfo(ctypes.Structure):
                 ("rows_light", ctypes.c_int64), ("rows_empty", ctypes.c_int64), ("nnz_a_heavy", ctypes.c_int64),
                 ("c_nnz_upper", ctypes.c_int64), ("n_batches", ctypes.c_int64), ("stage_elems", ctypes.c_int64),
                 ("workspace_bytes", ctypes.c_int64), ("light_bin_rows", ctypes.c_int64 * 8),
-                ("launches", ctypes.c_int64)]
+                ("launches", ctypes.c_int64), ("level0_direct", ctypes.c_int64)]
 
 
 class ExecStats(ctypes.Structure):

@@ -13,6 +13,7 @@
 #include "gm_k1_analysis.cuh"
 #include "gm_k3_light.cuh"
 #include "gm_k4_expand.cuh"
+#include "gm_k4_direct.cuh"
 #include "gm_k5_multisplit.cuh"
 #include "gm_k6_accumulate.cuh"
 #include "gm_k7_gather.cuh"
@@ -147,6 +148,12 @@ struct gm_plan {
   int64_t* seg_off = nullptr;      // n_seg + 1
   int64_t* seg_bstart = nullptr;   // n_seg
   int64_t* seg_j = nullptr;        // n_seg
+  int32_t* seg_brow = nullptr;     // n_seg: row of B the segment copies
+  uint32_t* child_bound = nullptr; // n_rows(B) x (F0 + 1): where each level-0 child starts inside a row of B
+  uint32_t* seg_prefix = nullptr;  // G: (segments of a batch + 1) x F0
+  uint32_t* seg_tile_sums = nullptr;
+  bool direct = false;             // the expansion writes the level-0 children itself
+  std::vector<int64_t> heavy_nz_off_host;
   int64_t* heavy_nz_off = nullptr; // nH + 1
   int32_t* sym_rows = nullptr;     // bins x nA
   int* sym_fill = nullptr;         // 8
@@ -329,18 +336,22 @@ static int build_plan(gm_plan* p, cudaStream_t st) {
     GM_TRY(plan_alloc(p, &p->seg_off, static_cast<size_t>(p->n_seg) + 1, st));
     GM_TRY(plan_alloc(p, &p->seg_bstart, static_cast<size_t>(p->n_seg) + 1, st));
     GM_TRY(plan_alloc(p, &p->seg_j, static_cast<size_t>(p->n_seg) + 1, st));
+    GM_TRY(plan_alloc(p, &p->seg_brow, static_cast<size_t>(p->n_seg) + 1, st));
     k1_heavy_scatter<<<grid_for(nA, 256, p->num_sms), 256, 0, st>>>(p->heavy_flag, heavy_pos, p->ip, A.row_ptr, nA,
                                                                    p->x_heavy, heavy_ip, heavy_nnz);
     exclusive_scan<i64, i64>(heavy_ip, p->heavy_base, nH, p->scan_tmp, nullptr, nullptr, nullptr, st);
     exclusive_scan<i64, i64>(heavy_nnz, p->heavy_nz_off, nH, p->scan_tmp, nullptr, nullptr, nullptr, st);
     k1_heavy_segments<<<grid_for(p->n_seg + 1, 256, p->num_sms, 32), 256, 0, st>>>(
         p->x_heavy, nH, p->heavy_nz_off, p->heavy_base, A.row_ptr, A.col_idx, p->nz_off, B.row_ptr, p->n_seg, p->seg_off,
-        p->seg_bstart, p->seg_j);
+        p->seg_bstart, p->seg_j, p->seg_brow);
     info.launches += 8;
     std::vector<int64_t> hb(static_cast<size_t>(nH) + 1);
     p->x_heavy_host.resize(static_cast<size_t>(nH));
     GM_CUDA(cudaMemcpyAsync(hb.data(), p->heavy_base, hb.size() * sizeof(int64_t), cudaMemcpyDeviceToHost, st));
     GM_CUDA(cudaMemcpyAsync(p->x_heavy_host.data(), p->x_heavy, static_cast<size_t>(nH) * sizeof(int32_t),
+                            cudaMemcpyDeviceToHost, st));
+    p->heavy_nz_off_host.resize(static_cast<size_t>(nH) + 1);
+    GM_CUDA(cudaMemcpyAsync(p->heavy_nz_off_host.data(), p->heavy_nz_off, (static_cast<size_t>(nH) + 1) * sizeof(int64_t),
                             cudaMemcpyDeviceToHost, st));
     GM_CUDA(cudaStreamSynchronize(st));
 
@@ -384,6 +395,29 @@ static int build_plan(gm_plan* p, cudaStream_t st) {
     const size_t n_tiles_max = static_cast<size_t>(info.stage_elems) / std::min({kExpandTile, kSplitTile, kGatherTile}) + 2;
     GM_TRY(plan_alloc(p, &p->tile_meta, n_tiles_max, st));
     GM_TRY(plan_alloc(p, &p->row_meta, n_tiles_max, st));
+    // The expansion writes the first level's children itself (see gm_k4_direct.cuh) unless asked to run that
+    // level as separate histogram and multisplit passes.
+    // That takes a row of F0 run starts per segment, which pays when segments are long compared with the
+    // fan-out (R-MAT products: ~1000 products per segment) and not when they are short (a clipped-Zipf pair
+    // with F0 = 256 and ~60 products per segment measured 3x slower that way).
+    const bool long_segments = info.products_heavy >= 2 * static_cast<i64>(prm.fanout[0]) * std::max<i64>(info.nnz_a_heavy, 1);
+    p->direct = prm.n_levels > 0 && prm.fanout[0] <= 256 &&
+                (p->opts.level0_multisplit == 2 || (p->opts.level0_multisplit == 0 && long_segments));
+    info.level0_direct = p->direct ? 1 : 0;
+    if (p->direct) {
+      const int F0 = prm.fanout[0];
+      i64 max_seg_b = 0;
+      for (const Batch& b : p->batches)
+        max_seg_b = std::max(max_seg_b, p->heavy_nz_off_host[static_cast<size_t>(b.h1)] - p->heavy_nz_off_host[static_cast<size_t>(b.h0)]);
+      GM_TRY(plan_alloc(p, &p->child_bound, static_cast<size_t>(B.n_rows) * static_cast<size_t>(F0 + 1) + 1, st));
+      GM_TRY(plan_alloc(p, &p->seg_prefix, (static_cast<size_t>(max_seg_b) + 1) * static_cast<size_t>(F0), st));
+      GM_TRY(plan_alloc(p, &p->seg_tile_sums, (static_cast<size_t>(max_seg_b) / kGTile + 2) * static_cast<size_t>(F0), st));
+      if (B.n_rows > 0) {
+        k_child_bounds<<<grid_for(B.n_rows * (F0 + 1), 256, p->num_sms, 32), 256, 0, st>>>(B.row_ptr, B.col_idx, B.n_rows, F0,
+                                                                                        prm.shift[0], p->child_bound);
+        ++info.launches;
+      }
+    }
     int64_t* tmp2 = nullptr;  // the per-batch scans can be longer than the ones above
     GM_TRY(plan_alloc(p, &tmp2, static_cast<size_t>(scan_tmp_elems(std::max<i64>({static_cast<i64>(n_chunks_max), nnzA, nA, 1}))), st));
     p->scan_tmp = tmp2;
@@ -553,8 +587,48 @@ static int heavy_batch_front(gm_plan* p, const Batch& b, HeavyBatchState<V>* hs,
   i64* off_nxt = p->level_off[1];
   k_rebase<<<grid_for(rows_b + 1, 256, p->num_sms), 256, 0, st>>>(p->heavy_base + b.h0, rows_b + 1, b.elem0, off_cur);
   ++p->stats.launches;
+  int cur = 0;
+  i64 n_par = rows_b;
+  int first_level = 0;
+  if (p->direct) {
+    // ---- run starts of every (segment, child) from counts alone, then the products straight into the children
+    const int F = prm.fanout[0];
+    const i64 seg0 = p->heavy_nz_off_host[static_cast<size_t>(b.h0)];
+    const i64 n_seg_b = p->heavy_nz_off_host[static_cast<size_t>(b.h1)] - seg0;
+    const i64 n_gt = (n_seg_b + kGTile - 1) / kGTile;
+    const i64 n_child = rows_b * F;
+    const unsigned ggrid = static_cast<unsigned>((n_gt + (256 / F) - 1) / (256 / F));
+    tm.begin(PhaseTimes::kHist, st);
+    k_g_tile_sums<<<ggrid, 256, 0, st>>>(p->seg_brow, seg0, n_seg_b, p->child_bound, F, p->seg_tile_sums);
+    k_g_scan_tiles<<<static_cast<unsigned>(F), 256, 0, st>>>(p->seg_tile_sums, n_gt, F);
+    k_g_write<<<ggrid, 256, 0, st>>>(p->seg_brow, seg0, n_seg_b, p->child_bound, F, p->seg_tile_sums, p->seg_prefix);
+    k_g_row_counts<<<grid_for(n_child, 256, p->num_sms, 32), 256, 0, st>>>(p->seg_prefix, p->heavy_nz_off + b.h0, seg0, rows_b, F,
+                                                                          p->counts);
+    p->stats.launches += 4;
+    tm.end(st);
+    tm.begin(PhaseTimes::kScan, st);
+    exclusive_scan<u32, i64>(p->counts, off_nxt, n_child, p->scan_tmp, nullptr, nullptr, nullptr, st);
+    p->stats.launches += 3;
+    tm.end(st);
+    tm.begin(PhaseTimes::kExpand, st);
+    const unsigned grid = static_cast<unsigned>((b.elems + kExpandTile - 1) / kExpandTile);
+    k_tile_bounds<<<grid_for(grid, 256, p->num_sms), 256, 0, st>>>(p->seg_off, p->n_seg, b.elem0, b.elems, kExpandTile,
+                                                                 p->tile_meta);
+    k_tile_bounds<<<grid_for(grid, 256, p->num_sms), 256, 0, st>>>(off_cur, rows_b, 0, b.elems, kExpandTile, p->row_meta);
+    k4_expand_direct<V><<<grid, kExpandThreads, 0, st>>>(
+        p->seg_off, p->seg_bstart, p->seg_j, p->seg_brow, p->tile_meta, static_cast<const V*>(p->A.vals), p->B.row_ptr,
+        p->B.col_idx, static_cast<const V*>(p->B.vals), b.elem0, b.elems, p->row_meta, off_cur, p->heavy_nz_off + b.h0, seg0, F,
+        prm.shift[0], off_nxt, p->seg_prefix, p->child_bound, p->stage_col[0], static_cast<V*>(p->stage_val[0]));
+    p->stats.launches += 3;
+    GM_CUDA(cudaGetLastError());
+    tm.end(st);
+    std::swap(off_cur, off_nxt);
+    n_par = n_child;
+    first_level = 1;
+  }
   // the expansion kernel counts the first level's (row, child) bins while it writes, unless asked not to
-  const bool fuse_hist = prm.n_levels > 0 && !p->opts.separate_histogram;
+  const bool fuse_hist = !p->direct && prm.n_levels > 0 && !p->opts.separate_histogram;
+  if (!p->direct) {
   tm.begin(PhaseTimes::kExpand, st);
   {
     static_assert(kExpandTile == kSplitTile, "the fused histogram shares the multisplit's tiles");
@@ -576,13 +650,12 @@ static int heavy_batch_front(gm_plan* p, const Batch& b, HeavyBatchState<V>* hs,
     GM_CUDA(cudaGetLastError());
   }
   tm.end(st);
-  int cur = 0;
-  i64 n_par = rows_b;
-  if (prm.n_levels > 0) {
+  }
+  if (prm.n_levels > first_level) {
     GM_CUDA(cudaFuncSetAttribute(k5_level<V, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                  static_cast<int>(split_smem_bytes<V>(true))));
   }
-  for (int l = 0; l < prm.n_levels; ++l) {
+  for (int l = first_level; l < prm.n_levels; ++l) {
     const int F = prm.fanout[l];
     const i64 n_child = n_par * F;
     const unsigned grid = static_cast<unsigned>((b.elems + kSplitTile - 1) / kSplitTile);

@@ -263,11 +263,34 @@ def test_config4_zipf_wide_columns_three_levels_sampled_rows():
 
 @pytest.mark.parametrize("separate", [0, 1])
 def test_fused_and_stand_alone_histogram_agree(separate):
-    # level-0 counts come either from the expansion kernel (default) or from the histogram kernel
+    # first level as separate passes over the staging buffer (Algorithm 5 as printed); its counts come either
+    # from the expansion kernel or from the histogram kernel
     A = gen.rmat(13, 16, seed=11, dtype=np.float32)
     C, info, stats = check_product(A, A, tau=512, chunk_width=512, max_fanout=4, separate_histogram=separate,
-                                   stage_elems=1 << 20)
-    assert info.params.n_levels == 2 and info.n_batches > 1
+                                   level0_multisplit=1, stage_elems=1 << 20)
+    assert info.params.n_levels == 2 and info.n_batches > 1 and info.level0_direct == 0
+
+
+@pytest.mark.parametrize("dtype,fanout,width", [(np.float32, 4, 512), (np.float64, 32, 256), (np.float32, 256, 32)])
+def test_expansion_straight_into_the_first_level(dtype, fanout, width):
+    # default path: the expansion kernel places every product in its level-0 child from counts alone.
+    # Several batches, one to three levels, and (narrow chunks with fan-out 256) tiles with more
+    # (segment, child) pairs than the per-tile table of run starts holds.
+    A = gen.rmat(13, 16, seed=11, dtype=dtype)
+    C, info, stats = check_product(A, A, tau=256, chunk_width=width, max_fanout=fanout, stage_elems=1 << 20,
+                                   level0_multisplit=2)
+    assert info.level0_direct == 1 and info.n_batches > 1 and info.params.n_levels >= 1
+
+
+def test_expansion_straight_into_the_first_level_short_rows_of_b():
+    # rows of B with 0 to 3 entries: tiles with thousands of segments, empty segments, heavy rows made of them
+    rng = np.random.default_rng(23)
+    B = random_csr(rng, 3000, 5000, 0.0004, np.float32)
+    A = random_csr(rng, 40, 3000, 0.6, np.float32)
+    C, info, stats = check_product(A, B, tau=64, chunk_width=256, max_fanout=4, level0_multisplit=2)
+    assert info.level0_direct == 1 and info.rows_heavy == 40
+    C, info, stats = check_product(A, B, tau=64, chunk_width=256, max_fanout=4)  # short segments: separate passes
+    assert info.level0_direct == 0
 
 
 @pytest.mark.parametrize("ctas", [1, 2, 4, 8])
