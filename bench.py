@@ -256,6 +256,8 @@ def main():
     ap.add_argument("--e2e-steps", type=int, default=2)
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--opt", action="append", default=[], metavar="FIELD=INT",
+                    help="set a field of gm_plan_opts (e.g. level0_multisplit=1, tau=4096); repeatable")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 1)
 
@@ -286,6 +288,11 @@ def main():
     dA = gm.DeviceCSR.from_host(A)
     dB = dA if B is A else gm.DeviceCSR.from_host(B)
     opts = gm.PlanOpts()
+    for kv in args.opt:
+        field, _, value = kv.partition("=")
+        if field not in dict(opts._fields_) or field == "reserved":
+            raise SystemExit(f"--opt: gm_plan_opts has no field '{field}'")
+        setattr(opts, field, int(value))
 
     def step(timing: bool):
         plan = gm.spgemm_plan(dA, dB, SMEM_BYTES, opts)
@@ -363,6 +370,7 @@ def main():
                    "products": products, "products_heavy": int(info.products_heavy), "nnz_c": int(nnz),
                    "rows_heavy": int(info.rows_heavy), "tau": int(tau), "chunk_width": int(info.params.chunk_width),
                    "levels": info.params.levels(), "batches": int(info.n_batches), "smem_bytes": SMEM_BYTES,
+                   "level0_direct": int(info.level0_direct), "plan_opts": args.opt,
                    "step": "gm_spgemm_plan + gm_spgemm_execute (C freed after each step)"},
         "roofline": roofline, "kernels": kt, "clocks": clocks, "gpu_launches": launches,
     }

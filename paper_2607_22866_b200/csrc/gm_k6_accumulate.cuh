@@ -242,7 +242,8 @@ __global__ void __launch_bounds__(kSmallWarps * 32) k6_small_chunks(
   const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
   const u32 wmask = static_cast<u32>(W - 1);
   const i64 n_groups = (n_chunks + 31) >> 5;
-  u64 sum_n = 0, sum_out = 0;
+  __shared__ u64 s_sum[kSmallWarps][2];  // statistics, kept out of the registers of the sort
+  if (lane == 0) { s_sum[w][0] = 0; s_sum[w][1] = 0; }
   // a warp looks at 32 consecutive chunks at a time and works through the small ones among them
   for (i64 g = static_cast<i64>(blockIdx.x) * kSmallWarps + w; g < n_groups; g += static_cast<i64>(gridDim.x) * kSmallWarps) {
     const i64 k = (g << 5) + lane;
@@ -268,13 +269,12 @@ __global__ void __launch_bounds__(kSmallWarps * 32) k6_small_chunks(
       else if (kSmallMaxPerLane == 8 || n <= 256) m = small_chunk<V, 8>(col, val, n, wmask, s_key[w], s_val[w], out);
       else if (kSmallMaxPerLane == 16 || n <= 512) m = small_chunk<V, (kSmallMaxPerLane >= 16 ? 16 : 8)>(col, val, n, wmask, s_key[w], s_val[w], out);
       else m = small_chunk<V, kSmallMaxPerLane>(col, val, n, wmask, s_key[w], s_val[w], out);
-      sum_n += static_cast<u64>(n);
-      sum_out += static_cast<u64>(m);
+      if (lane == 0) { s_sum[w][0] += static_cast<u64>(n); s_sum[w][1] += static_cast<u64>(m); }
     }
   }
-  if (lane == 0 && sum_n) {
-    atomicAdd(&totals[0], sum_n);
-    atomicAdd(&totals[1], sum_out);
+  if (lane == 0 && s_sum[w][0]) {
+    atomicAdd(&totals[0], s_sum[w][0]);
+    atomicAdd(&totals[1], s_sum[w][1]);
   }
 }
 
