@@ -11,6 +11,10 @@ namespace gm {
 
 constexpr int kGatherThreads = 256;
 constexpr int kGatherTile = 4096;
+#ifndef GM_GATHER_BATCH
+#define GM_GATHER_BATCH 4
+#endif
+constexpr int kGatherBatch = GM_GATHER_BATCH;  // positions a thread has in flight
 constexpr int kGatherChunkCap = 1024;  // chunks staged in shared memory per tile; more -> per-element search
 
 template <typename V>
@@ -38,25 +42,43 @@ __global__ void __launch_bounds__(kGatherThreads) k7_gather(
       }
     }
     __syncthreads();
-    // each thread walks kGatherTile / kGatherThreads positions strided by the block; its chunk index only grows
+    // each thread walks kGatherTile / kGatherThreads positions strided by the block; its chunk index only grows.
+    // Positions are taken kGatherBatch at a time, all loads before the first store, so that a thread has that
+    // many independent loads in flight (one at a time left the kernel waiting on memory at full occupancy).
     int cur = 0;
-#pragma unroll 4
-    for (int q = threadIdx.x; q < tn; q += kGatherThreads) {
-      // last chunk whose start is <= q (empty chunks share a start with their successor and are skipped)
-      int lo = cur, hi = n_k - 1;
-      while (lo < hi) {
-        const int mid = lo + ((hi - lo + 1) >> 1);
-        if (s_rel[mid] <= q) lo = mid; else hi = mid - 1;
+    for (int q0 = threadIdx.x; q0 < tn; q0 += kGatherBatch * kGatherThreads) {
+      i64 dst[kGatherBatch];
+      int32_t col[kGatherBatch];
+      V val[kGatherBatch];
+#pragma unroll
+      for (int u = 0; u < kGatherBatch; ++u) {
+        const int q = q0 + u * kGatherThreads;
+        dst[u] = -1;
+        if (q < tn) {
+          // last chunk whose start is <= q (empty chunks share a start with their successor and are skipped)
+          int lo = cur, hi = n_k - 1;
+          while (lo < hi) {
+            const int mid = lo + ((hi - lo + 1) >> 1);
+            if (s_rel[mid] <= q) lo = mid; else hi = mid - 1;
+          }
+          cur = lo;
+          const i64 r = static_cast<i64>(q) - s_rel[cur];
+          dst[u] = s_dst[cur] + r;
+          const i64 src = s_src[cur] + r;
+          col[u] = s_col_in[src];
+          val[u] = s_val_in[src];
+        }
       }
-      cur = lo;
-      const i64 r = static_cast<i64>(q) - s_rel[cur];
-      const i64 dst = s_dst[cur] + r;
-      if (dst < c_capacity) {
-        const i64 src = s_src[cur] + r;
-        c_col[dst] = s_col_in[src];
-        c_val[dst] = s_val_in[src];
-      } else {
-        dev_set_error(err, kDevCapacity);
+#pragma unroll
+      for (int u = 0; u < kGatherBatch; ++u) {
+        if (dst[u] >= 0) {
+          if (dst[u] < c_capacity) {
+            c_col[dst[u]] = col[u];
+            c_val[dst[u]] = val[u];
+          } else {
+            dev_set_error(err, kDevCapacity);
+          }
+        }
       }
     }
   } else {
