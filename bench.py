@@ -40,7 +40,8 @@ DEFAULT_CONFIG = 2  # R-MAT scale 20, edge factor 16, fp32: the largest fp32 pow
 # launch, measured on a scaled-down case of the same kernels (R-MAT scale 17, 1.09 G products per step: see
 # profiles/dram_traffic_rmat17_f32.md).  Traffic grows in proportion to the products processed, so a full-size
 # launch is the algorithmic figure times this ratio.
-TRAFFIC_RATIO = {"k4_expand": 1.03, "k5b_multisplit": 0.99, "k6_small_chunks": 0.73, "k6_accumulate": 1.01, "k7_gather": 0.99}
+TRAFFIC_RATIO = {"k4_expand": 1.03, "k5a_histogram": 0.34, "k5b_multisplit": 0.99, "k6_small_chunks": 0.73, "k6_accumulate": 1.01,
+                 "k7_gather": 0.99}
 
 
 def _peaks():
