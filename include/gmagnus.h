@@ -71,9 +71,10 @@ typedef struct gm_plan_opts {
   int32_t acc_ctas_per_sm; /* 1, 2, 4 or 8: how many chunk accumulators share one SM (sets W)  */
   int64_t stage_elems;     /* capacity, in intermediate products, of each staging half-buffer  */
   int64_t c_capacity;      /* room, in entries, reserved for C when heavy rows need > 1 batch  */
-  int32_t separate_histogram; /* 1: always run the stand-alone histogram kernel per level      */
+  int32_t separate_histogram; /* 1: always run the stand-alone histogram kernel per level (otherwise a
+                              first level that runs as separate passes is counted by the expansion) */
   int32_t validate_inputs; /* 1: check row_ptr / col_idx of A and B on the device first        */
-  int32_t single_stream;   /* 1: do not overlap the light and heavy paths on forked streams    */
+  int32_t single_stream;   /* accepted and ignored: all work of a call runs on the caller's stream */
   int32_t level0_multisplit; /* first multisplit level: 1 = separate histogram and multisplit passes over
                               the staging buffer (Algorithm 5 as printed); 2 = the expansion kernel writes
                               the first level's children itself; 0 (default) = the latter when the heavy
@@ -174,13 +175,15 @@ int gm_spgemm_plan_ex(const gm_csr* A, const gm_csr* B, size_t smem_bytes,
 
 /* The rest of Algorithm 3: light rows by Gustavson's method with a shared-memory hash accumulator
  * (symbolic, then numeric); heavy rows, batch by batch, through the expansion (outer-product)
- * kernel (Algorithm 4), one histogram + multisplit (Algorithm 5) per level, the dense
- * chunk-accumulate kernel (which compacts every chunk in place and counts its entries) and, once
+ * kernel (Algorithm 4), one histogram + multisplit (Algorithm 5) per level (by default the first
+ * level is done by the expansion kernel itself, see gm_plan_opts.level0_multisplit), the
+ * chunk-accumulate kernels (small chunks by a one-warp sort, the others in the dense shared-memory
+ * accumulator of Section III-E; every chunk is compacted in place and its entries counted) and, once
  * C.row_ptr is known by prefix sums over the per-row counts, the gather of the chunks into C.
  *   C_out  host struct filled with device pointers allocated through the allocator hook;
  *          C_out->nnz is exact.  Release with gm_csr_free.
- * Work is enqueued on `cuda_stream` (and internal streams forked from and joined back to it); the
- * call returns after synchronising that stream, because nnz(C) is needed on the host.
+ * Work is enqueued on `cuda_stream`; the call returns after synchronising that stream, because nnz(C)
+ * is needed on the host.
  * A plan can be executed any number of times (values of A and B may change in between, their
  * structure may not).  Two executes of the same plan must not overlap.
  * Errors: GM_ERR_CAPACITY (C did not fit the reserved room; only possible when the heavy rows
