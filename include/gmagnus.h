@@ -195,7 +195,10 @@ int gm_spgemm_execute(gm_plan* plan, void* cuda_stream, gm_csr* C_out);
  * device, plans, executes, and copies C back.  C_host->row_ptr / col_idx / vals must point to
  * caller-owned buffers with room for n_rows + 1 / c_capacity / c_capacity entries; on return
  * C_host->nnz is set.  If nnz(C) > c_capacity only row_ptr is copied and GM_ERR_CAPACITY is
- * returned (C_host->nnz then tells the room needed).  Synchronous. */
+ * returned (C_host->nnz then tells the room needed).  Synchronous.  When the heavy rows take several
+ * batches, the rows of every batch (its light rows included) are finished and copied out while the next
+ * batch computes, so the copy of C overlaps the computation; the buffers hold valid entries only after
+ * the call has returned GM_OK. */
 int gm_spgemm_host(const gm_csr* A_host, const gm_csr* B_host, size_t smem_bytes,
                    const gm_plan_opts* opts, gm_csr* C_host, int64_t c_capacity);
 

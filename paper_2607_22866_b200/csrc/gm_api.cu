@@ -123,6 +123,17 @@ struct PhaseTimes {
 
 }  // namespace gm
 
+// Where gm_spgemm_host wants C: entries are copied to the host batch by batch, while later batches compute.
+struct HostSink {
+  int32_t* h_col = nullptr;
+  void* h_val = nullptr;
+  int64_t capacity = 0;          // entries the host buffers hold
+  cudaStream_t copy_stream = nullptr;
+  int64_t* h_totals = nullptr;   // pinned: entries of C up to the end of each batch
+  std::vector<cudaEvent_t> events;
+  int64_t copied = 0;            // entries already on their way to the host
+};
+
 struct gm_plan {
   gm_csr A{}, B{};
   int sv = 4;
@@ -177,6 +188,7 @@ struct gm_plan {
   gm::TileMeta* row_meta = nullptr;   // per tile of the expansion kernel: heavy rows it touches (fused histogram)
   gm::TileMeta* tile_meta = nullptr;  // per tile of the expansion / multisplit kernels: groups it touches
   gm::PhaseTimes times;
+  HostSink* sink = nullptr;        // set by gm_spgemm_host for the duration of one execute
 };
 
 namespace gm {
@@ -755,18 +767,20 @@ static int execute_t(gm_plan* p, cudaStream_t st, gm_csr* C) {
     i64 run = 0;
     for (int b = p->bins.n_bins - 1; b >= 0; --b) { run += info.light_bin_rows[b]; num_upper[b] = run; }
   }
-  auto light_numeric = [&](i64 capacity) -> int {
+  // numeric pass of the light rows in [r0, r1) (all of them by default)
+  auto light_numeric_range = [&](i64 capacity, i64 r0, i64 r1) -> int {
     tm.begin(PhaseTimes::kLightNum, st);
-    if (info.rows_light > 0) {
+    if (info.rows_light > 0 && r1 > r0) {
       GM_CUDA(cudaMemsetAsync(p->num_fill, 0, 8 * sizeof(int), st));
-      k1_bin_rows<int32_t><<<static_cast<unsigned>((nA + 255) / 256), 256, 0, st>>>(p->row_nnz, p->heavy_flag, nA, p->bins,
-                                                                                    std::max<i64>(nA, 1), p->num_fill, p->num_rows);
+      k1_bin_rows<int32_t><<<static_cast<unsigned>((r1 - r0 + 255) / 256), 256, 0, st>>>(
+          p->row_nnz + r0, p->heavy_flag + r0, r1 - r0, p->bins, std::max<i64>(nA, 1), p->num_fill, p->num_rows, r0);
       ++p->stats.launches;
       GM_TRY((launch_light<V, true>(p, p->num_rows, p->num_fill, num_upper, c_row_ptr, c_col, c_val, capacity, st)));
     }
     tm.end(st);
     return GM_OK;
   };
+  auto light_numeric = [&](i64 capacity) -> int { return light_numeric_range(capacity, 0, nA); };
 
   const size_t n_batches = p->batches.size();
   i64 capacity = 0;
@@ -840,8 +854,34 @@ static int execute_t(gm_plan* p, cudaStream_t st, gm_csr* C) {
       tm.begin(PhaseTimes::kAccSym, st);
       GM_TRY_C((launch_gather<V>(p, b, hs, c_row_ptr, c_col, c_val, capacity, st)));
       tm.end(st);
+      if (HostSink* sk = p->sink) {
+        // The caller wants C on the host: finish rows [r0, r1) now (their light rows too), note how many entries
+        // of C that makes, and send the previous batch's entries on their way while this batch computes.
+        GM_TRY_C(light_numeric_range(capacity, r0, r1));
+        if (sk->events.size() <= bi) {
+          cudaEvent_t ev = nullptr;
+          if (cudaEventCreateWithFlags(&ev, cudaEventDisableTiming) != cudaSuccess) { cleanup(); return fail(GM_ERR_CUDA, "event creation failed"); }
+          sk->events.push_back(ev);
+        }
+        cudaMemcpyAsync(&sk->h_totals[bi], p->c_total, sizeof(i64), cudaMemcpyDeviceToHost, st);
+        cudaEventRecord(sk->events[bi], st);
+        auto send = [&](size_t done) {
+          if (cudaEventSynchronize(sk->events[done]) != cudaSuccess) return;
+          const i64 end = std::min<i64>(sk->h_totals[done], sk->capacity);
+          if (end > sk->copied) {
+            cudaStreamWaitEvent(sk->copy_stream, sk->events[done], 0);
+            cudaMemcpyAsync(sk->h_col + sk->copied, c_col + sk->copied, static_cast<size_t>(end - sk->copied) * sizeof(int32_t),
+                            cudaMemcpyDeviceToHost, sk->copy_stream);
+            cudaMemcpyAsync(static_cast<V*>(sk->h_val) + sk->copied, c_val + sk->copied,
+                            static_cast<size_t>(end - sk->copied) * sizeof(V), cudaMemcpyDeviceToHost, sk->copy_stream);
+            sk->copied = end;
+          }
+        };
+        if (bi > 0) send(bi - 1);
+        if (bi + 1 == n_batches) send(bi);
+      }
     }
-    GM_TRY_C(light_numeric(capacity));
+    if (!p->sink) GM_TRY_C(light_numeric(capacity));
     if (cudaMemcpyAsync(&total, p->c_total, sizeof(i64), cudaMemcpyDeviceToHost, st) != cudaSuccess) {
       cleanup();
       return fail(GM_ERR_CUDA, "copy of nnz(C) failed");
@@ -1028,7 +1068,19 @@ int gm_spgemm_host(const gm_csr* A_host, const gm_csr* B_host, size_t smem_bytes
   rc = upload(A_host, &dev[0]);
   if (rc == GM_OK) rc = upload(B_host, &dev[1]);
   if (rc == GM_OK) rc = gm_spgemm_plan_ex(&dev[0], &dev[1], smem_bytes, opts, st, &plan);
+  // With several batches, C's entries travel to the host batch by batch while later batches compute.
+  HostSink sink;
+  bool use_sink = false;
+  if (rc == GM_OK && plan->batches.size() > 1 && C_host->col_idx && C_host->vals && c_capacity > 0) {
+    sink.h_col = const_cast<int32_t*>(C_host->col_idx);
+    sink.h_val = const_cast<void*>(C_host->vals);
+    sink.capacity = c_capacity;
+    use_sink = cudaStreamCreateWithFlags(&sink.copy_stream, cudaStreamNonBlocking) == cudaSuccess &&
+               cudaMallocHost(reinterpret_cast<void**>(&sink.h_totals), plan->batches.size() * sizeof(int64_t)) == cudaSuccess;
+    if (use_sink) plan->sink = &sink;
+  }
   if (rc == GM_OK) rc = gm_spgemm_execute(plan, st, &C);
+  if (plan) plan->sink = nullptr;
   if (rc == GM_OK) {
     C_host->n_rows = C.n_rows;
     C_host->n_cols = C.n_cols;
@@ -1042,13 +1094,18 @@ int gm_spgemm_host(const gm_csr* A_host, const gm_csr* B_host, size_t smem_bytes
       if (!C_host->col_idx || !C_host->vals) {
         rc = fail(GM_ERR_INVALID_ARG, "C_host->col_idx / vals are null");
       } else {
-        e = cudaMemcpyAsync(const_cast<int32_t*>(C_host->col_idx), C.col_idx, static_cast<size_t>(C.nnz) * 4,
-                            cudaMemcpyDeviceToHost, st);
-        if (e == cudaSuccess)
-          e = cudaMemcpyAsync(const_cast<void*>(C_host->vals), C.vals, static_cast<size_t>(C.nnz) * sv,
-                              cudaMemcpyDeviceToHost, st);
+        const int64_t done = use_sink ? sink.copied : 0;  // entries the batches have already sent
+        if (C.nnz > done) {
+          e = cudaMemcpyAsync(const_cast<int32_t*>(C_host->col_idx) + done, C.col_idx + done,
+                              static_cast<size_t>(C.nnz - done) * 4, cudaMemcpyDeviceToHost, st);
+          if (e == cudaSuccess)
+            e = cudaMemcpyAsync(static_cast<char*>(const_cast<void*>(C_host->vals)) + static_cast<size_t>(done) * sv,
+                                static_cast<const char*>(C.vals) + static_cast<size_t>(done) * sv,
+                                static_cast<size_t>(C.nnz - done) * sv, cudaMemcpyDeviceToHost, st);
+        }
       }
     }
+    if (use_sink && cudaStreamSynchronize(sink.copy_stream) != cudaSuccess && e == cudaSuccess) e = cudaErrorUnknown;
     cudaError_t e2 = cudaStreamSynchronize(st);
     if (rc == GM_OK && (e != cudaSuccess || e2 != cudaSuccess)) rc = fail(GM_ERR_CUDA, "copy of C to the host failed");
     dev_free(const_cast<int64_t*>(C.row_ptr), st);
@@ -1061,6 +1118,12 @@ int gm_spgemm_host(const gm_csr* A_host, const gm_csr* B_host, size_t smem_bytes
   }
   for (void* q : tmp) dev_free(q, st);
   cudaStreamSynchronize(st);
+  if (sink.copy_stream) {
+    cudaStreamSynchronize(sink.copy_stream);
+    cudaStreamDestroy(sink.copy_stream);
+  }
+  for (cudaEvent_t ev : sink.events) cudaEventDestroy(ev);
+  if (sink.h_totals) cudaFreeHost(sink.h_totals);
   cudaStreamDestroy(st);
   return rc;
 }

@@ -120,7 +120,8 @@ __global__ void k1_heavy_segments(const int32_t* __restrict__ x_heavy, i64 n_hea
 template <typename SizeT>
 __global__ void __launch_bounds__(256) k1_bin_rows(const SizeT* __restrict__ size, const int32_t* __restrict__ skip,
                                                    i64 n_rows, LightBins lb, i64 bin_stride,
-                                                   int* __restrict__ bin_fill, int32_t* __restrict__ rows_out) {
+                                                   int* __restrict__ bin_fill, int32_t* __restrict__ rows_out,
+                                                   i64 row0 = 0) {  // size/skip start at row row0; rows_out gets global ids
   __shared__ int s_cnt[kMaxLightBins];
   __shared__ int s_base[kMaxLightBins];
   const i64 i = static_cast<i64>(blockIdx.x) * blockDim.x + threadIdx.x;
@@ -148,7 +149,7 @@ __global__ void __launch_bounds__(256) k1_bin_rows(const SizeT* __restrict__ siz
   }
   __syncthreads();
   if (bin >= 0)
-    rows_out[bin * bin_stride + s_base[bin] + s_warp[warp][bin] + rank] = static_cast<int32_t>(i);
+    rows_out[bin * bin_stride + s_base[bin] + s_warp[warp][bin] + rank] = static_cast<int32_t>(row0 + i);
 }
 
 }  // namespace gm

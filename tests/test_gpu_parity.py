@@ -214,6 +214,38 @@ def test_host_entry_point():
     assert ei.value.status == -6
 
 
+@pytest.mark.parametrize("dtype", [np.float32, np.float64])
+def test_host_entry_point_streams_batches_to_the_host(dtype):
+    # several batches: every batch's rows (light ones included) are finished and copied out while the next
+    # batch computes; pinned and pageable destinations, and a destination that is too small
+    import paper_2607_22866_b200 as gm
+    A = gen.rmat(12, 16, seed=9, dtype=dtype)
+    ref = oracle.spgemm(A, A)
+    o = gm.PlanOpts(); o.tau = 128; o.stage_elems = 1 << 17
+    tol = 1e-5 if dtype == np.float32 else 1e-12
+    for pinned in (False, True):
+        rp = np.empty(A.n_rows + 1, np.int64)
+        if pinned:
+            tcol = torch.empty(ref.nnz + 7, dtype=torch.int32, pin_memory=True)
+            tval = torch.empty(ref.nnz + 7, dtype=torch.float32 if dtype == np.float32 else torch.float64, pin_memory=True)
+            col, val = tcol.numpy(), tval.numpy()
+        else:
+            col = np.empty(ref.nnz + 7, np.int32)
+            val = np.empty(ref.nnz + 7, dtype)
+        col[:] = -1
+        nnz = gm.spgemm_host(A, A, rp, col, val, opts=o)
+        assert nnz == ref.nnz and np.array_equal(rp, ref.row_ptr) and np.array_equal(col[:nnz], ref.col)
+        assert np.all(np.abs(val[:nnz].astype(np.float64) - ref.val) <= tol * ref.abs)
+        assert np.all(col[nnz:] == -1)
+    dA = gm.DeviceCSR.from_host(A)
+    plan = gm.spgemm_plan(dA, dA, 232448, o)
+    assert plan.info().n_batches > 3
+    plan.destroy()
+    with pytest.raises(gm.GmError) as ei:
+        gm.spgemm_host(A, A, rp, col[:ref.nnz // 2], val[:ref.nnz // 2], opts=o)
+    assert ei.value.status == -6
+
+
 def _check_sampled_rows(A, B, n_random=200, n_heavy=60, **opts):
     """Full-size check in the launch configuration the benchmark times: structure and values of
     sampled rows (random rows, the heaviest rows, random heavy rows) against the row-range oracle,
