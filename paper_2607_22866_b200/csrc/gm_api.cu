@@ -413,8 +413,11 @@ static int build_plan(gm_plan* p, cudaStream_t st) {
     // fan-out (R-MAT products: ~1000 products per segment) and not when they are short (a clipped-Zipf pair
     // with F0 = 256 and ~60 products per segment measured 3x slower that way).
     const bool long_segments = info.products_heavy >= 2 * static_cast<i64>(prm.fanout[0]) * std::max<i64>(info.nnz_a_heavy, 1);
+    // ... and a table of F0 + 1 boundaries per row of B, which must stay small next to the staging buffers
+    const i64 bound_bytes = B.n_rows * static_cast<i64>(prm.fanout[0] + 1) * 4;
+    const bool bounds_fit = bound_bytes <= std::max<i64>(i64{1} << 30, static_cast<i64>(se) * (4 + p->sv));
     p->direct = prm.n_levels > 0 && prm.fanout[0] <= 256 &&
-                (p->opts.level0_multisplit == 2 || (p->opts.level0_multisplit == 0 && long_segments));
+                (p->opts.level0_multisplit == 2 || (p->opts.level0_multisplit == 0 && long_segments && bounds_fit));
     info.level0_direct = p->direct ? 1 : 0;
     if (p->direct) {
       const int F0 = prm.fanout[0];
