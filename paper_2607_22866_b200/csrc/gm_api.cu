@@ -162,6 +162,7 @@ struct gm_plan {
   int32_t* seg_brow = nullptr;     // n_seg: row of B the segment copies
   uint32_t* child_bound = nullptr; // n_rows(B) x (F0 + 1): where each level-0 child starts inside a row of B
   uint32_t* seg_prefix = nullptr;  // G: (segments of a batch + 1) x F0
+  uint32_t* seg_h = nullptr;       // H: segments of a batch x F0 (G minus the child boundary of the segment's row of B)
   uint32_t* seg_tile_sums = nullptr;
   bool direct = false;             // the expansion writes the level-0 children itself
   std::vector<int64_t> heavy_nz_off_host;
@@ -426,6 +427,7 @@ static int build_plan(gm_plan* p, cudaStream_t st) {
         max_seg_b = std::max(max_seg_b, p->heavy_nz_off_host[static_cast<size_t>(b.h1)] - p->heavy_nz_off_host[static_cast<size_t>(b.h0)]);
       GM_TRY(plan_alloc(p, &p->child_bound, static_cast<size_t>(B.n_rows) * static_cast<size_t>(F0 + 1) + 1, st));
       GM_TRY(plan_alloc(p, &p->seg_prefix, (static_cast<size_t>(max_seg_b) + 1) * static_cast<size_t>(F0), st));
+      GM_TRY(plan_alloc(p, &p->seg_h, (static_cast<size_t>(max_seg_b) + 1) * static_cast<size_t>(F0), st));
       GM_TRY(plan_alloc(p, &p->seg_tile_sums, (static_cast<size_t>(max_seg_b) / kGTile + 2) * static_cast<size_t>(F0), st));
       if (B.n_rows > 0) {
         k_child_bounds<<<grid_for(B.n_rows * (F0 + 1), 256, p->num_sms, 32), 256, 0, st>>>(B.row_ptr, B.col_idx, B.n_rows, F0,
@@ -616,14 +618,18 @@ static int heavy_batch_front(gm_plan* p, const Batch& b, HeavyBatchState<V>* hs,
     tm.begin(PhaseTimes::kHist, st);
     k_g_tile_sums<<<ggrid, 256, 0, st>>>(p->seg_brow, seg0, n_seg_b, p->child_bound, F, p->seg_tile_sums);
     k_g_scan_tiles<<<static_cast<unsigned>(F), 256, 0, st>>>(p->seg_tile_sums, n_gt, F);
-    k_g_write<<<ggrid, 256, 0, st>>>(p->seg_brow, seg0, n_seg_b, p->child_bound, F, p->seg_tile_sums, p->seg_prefix);
+    k_g_write<<<ggrid, 256, 0, st>>>(p->seg_brow, seg0, n_seg_b, p->child_bound, F, p->seg_tile_sums, p->seg_prefix, p->seg_h);
     k_g_row_counts<<<grid_for(n_child, 256, p->num_sms, 32), 256, 0, st>>>(p->seg_prefix, p->heavy_nz_off + b.h0, seg0, rows_b, F,
                                                                           p->counts);
     p->stats.launches += 4;
     tm.end(st);
     tm.begin(PhaseTimes::kScan, st);
     exclusive_scan<u32, i64>(p->counts, off_nxt, n_child, p->scan_tmp, nullptr, nullptr, nullptr, st);
-    p->stats.launches += 3;
+    // (the cursor array of the multisplit is free in this mode: it holds R)
+    u32* const row_base = reinterpret_cast<u32*>(p->cursor);
+    k_g_row_base<<<grid_for(n_child, 256, p->num_sms, 32), 256, 0, st>>>(p->seg_prefix, p->heavy_nz_off + b.h0, seg0, rows_b, F,
+                                                                        off_nxt, row_base);
+    p->stats.launches += 4;
     tm.end(st);
     tm.begin(PhaseTimes::kExpand, st);
     const unsigned grid = static_cast<unsigned>((b.elems + kExpandTile - 1) / kExpandTile);
@@ -631,9 +637,9 @@ static int heavy_batch_front(gm_plan* p, const Batch& b, HeavyBatchState<V>* hs,
                                                                  p->tile_meta);
     k_tile_bounds<<<grid_for(grid, 256, p->num_sms), 256, 0, st>>>(off_cur, rows_b, 0, b.elems, kExpandTile, p->row_meta);
     k4_expand_direct<V><<<grid, kExpandThreads, 0, st>>>(
-        p->seg_off, p->seg_bstart, p->seg_j, p->seg_brow, p->tile_meta, static_cast<const V*>(p->A.vals), p->B.row_ptr,
-        p->B.col_idx, static_cast<const V*>(p->B.vals), b.elem0, b.elems, p->row_meta, off_cur, p->heavy_nz_off + b.h0, seg0, F,
-        prm.shift[0], off_nxt, p->seg_prefix, p->child_bound, p->stage_col[0], static_cast<V*>(p->stage_val[0]));
+        p->seg_off, p->seg_bstart, p->seg_j, p->tile_meta, static_cast<const V*>(p->A.vals), p->B.col_idx,
+        static_cast<const V*>(p->B.vals), b.elem0, b.elems, p->row_meta, off_cur, seg0, F, prm.shift[0], row_base, p->seg_h,
+        p->stage_col[0], static_cast<V*>(p->stage_val[0]));
     p->stats.launches += 3;
     GM_CUDA(cudaGetLastError());
     tm.end(st);

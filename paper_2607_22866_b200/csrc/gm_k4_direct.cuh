@@ -12,8 +12,12 @@
 // first level.  Deeper levels run as in Algorithm 5.
 //
 //   k_child_bounds   (plan)   bound[k][c], c = 0..F, for every row of B
-//   k_g_tile_sums, k_g_scan_tiles, k_g_write   (per batch)   G[s][c] = sum of cnt[s'][c] over the batch's segments s' < s
+//   k_g_tile_sums, k_g_scan_tiles, k_g_write   (per batch)   G[s][c] = sum of cnt[s'][c] over the batch's segments s' < s,
+//                                                             and H[s][c] = G[s][c] - bound[k_s][c]
 //   k_g_row_counts   (per batch)   (row, child) counts, whose exclusive scan is child_off
+//   k_g_row_base     (per batch)   R[row][c] = child_off[row][c] - G[first segment of the row][c]
+// so that the product at position i of B[k_s,:] (child c) goes to R[row][c] + H[s][c] + i  (32-bit wrap-around
+// arithmetic; the result is a position inside the batch).
 //   k4_expand_direct (per batch)   the products, in place
 #pragma once
 #include "gm_common.cuh"
@@ -76,7 +80,7 @@ __global__ void __launch_bounds__(256) k_g_scan_tiles(u32* __restrict__ tile_sum
 // G[s * F + c] for s = 0..n_seg_b (the last row holds the batch's totals per child).
 __global__ void __launch_bounds__(256) k_g_write(const int32_t* __restrict__ seg_brow, i64 seg0, i64 n_seg_b,
                                                  const u32* __restrict__ bound, int F, const u32* __restrict__ tile_sums,
-                                                 u32* __restrict__ G) {
+                                                 u32* __restrict__ G, u32* __restrict__ H) {
   const int c = threadIdx.x & (F - 1);
   const i64 tile = static_cast<i64>(blockIdx.x) * (256 / F) + threadIdx.x / F;
   const i64 s_begin = tile * kGTile;
@@ -84,9 +88,11 @@ __global__ void __launch_bounds__(256) k_g_write(const int32_t* __restrict__ seg
   const i64 s_end = min(n_seg_b, s_begin + kGTile);
   u32 run = tile_sums[tile * F + c];
   for (i64 s = s_begin; s < s_end; ++s) {
-    G[s * F + c] = run;
     const u32* bp = bound + static_cast<i64>(seg_brow[seg0 + s]) * (F + 1) + c;
-    run += bp[1] - bp[0];
+    const u32 b0 = bp[0];
+    G[s * F + c] = run;
+    H[s * F + c] = run - b0;
+    run += bp[1] - b0;
   }
   if (s_end == n_seg_b) G[n_seg_b * F + c] = run;
 }
@@ -102,19 +108,28 @@ __global__ void k_g_row_counts(const u32* __restrict__ G, const i64* __restrict_
   }
 }
 
+// R[r * F + c] = child_off[r * F + c] - G[first segment of row r][c]  (mod 2^32)
+__global__ void k_g_row_base(const u32* __restrict__ G, const i64* __restrict__ row_seg, i64 seg0, i64 n_rows_b, int F,
+                             const i64* __restrict__ child_off, u32* __restrict__ R) {
+  const i64 n = n_rows_b * F;
+  for (i64 i = static_cast<i64>(blockIdx.x) * blockDim.x + threadIdx.x; i < n; i += static_cast<i64>(gridDim.x) * blockDim.x) {
+    const i64 r = i / F;
+    const int c = static_cast<int>(i - r * F);
+    R[i] = static_cast<u32>(child_off[i]) - G[(row_seg[r] - seg0) * F + c];
+  }
+}
+
 template <typename V>
 __global__ void __launch_bounds__(kExpandThreads) k4_expand_direct(
     const i64* __restrict__ seg_off, const i64* __restrict__ seg_bstart, const i64* __restrict__ seg_j,
-    const int32_t* __restrict__ seg_brow,
     const TileMeta* __restrict__ tile_meta,  // per tile: first segment and number of segments
-    const V* __restrict__ a_val, const i64* __restrict__ b_row_ptr, const int32_t* __restrict__ b_col,
-    const V* __restrict__ b_val,
+    const V* __restrict__ a_val, const int32_t* __restrict__ b_col, const V* __restrict__ b_val,
     i64 elem0, i64 n_elems,  // first product of the batch (global heavy numbering), batch size
     const TileMeta* __restrict__ row_meta, const i64* __restrict__ row_off,  // the batch's rows: tile records, product offsets
-    const i64* __restrict__ row_seg,  // first segment (global numbering) of every row of the batch, and one past the last
     i64 seg0,                          // first segment of the batch
-    int F, int shift, const i64* __restrict__ child_off,  // n_rows_b * F + 1 offsets of the level-0 children
-    const u32* __restrict__ G, const u32* __restrict__ bound,
+    int F, int shift,
+    const u32* __restrict__ R,  // (row of the batch, child): child_off - G at the row's first segment
+    const u32* __restrict__ H,  // (segment of the batch, child): G - bound
     int32_t* __restrict__ y_col, V* __restrict__ y_val) {
   __shared__ int s_tq[kDirectTableCap];  // (segment in tile, child) -> destination minus tile position
   __shared__ int s_roff[kExpandHistParents + 1];
@@ -148,13 +163,11 @@ __global__ void __launch_bounds__(kExpandThreads) k4_expand_direct(
     }
     return last_le(row_off, rm.first, rm.first + rm.n - 1, t0 + q) - rm.first;
   };
-  // final position of the product at tile position q, of segment s (global numbering), row `par`, child c
+  // final position of the product at tile position q, of segment s (global numbering), row `par`, child c:
+  // a segment starts at the beginning of its row of B, so the product's index in that row is p0 + q - seg_off[s]
   auto dst_global = [&](i64 s, i64 par, u32 c, int q) -> i64 {
-    const i64 p = rm.first + par;
-    const i64 brow = seg_brow[s];
-    const u32 before = G[(s - seg0) * F + c] - G[(row_seg[p] - seg0) * F + c];
-    return child_off[p * F + c] + static_cast<i64>(before) - static_cast<i64>(bound[brow * (F + 1) + c]) +
-           (seg_bstart[s] - b_row_ptr[brow]) + (p0 + q - seg_off[s]);
+    const u32 d = R[(rm.first + par) * F + c] + H[(s - seg0) * F + c] + static_cast<u32>(p0 + q - seg_off[s]);
+    return static_cast<i64>(d);
   };
 
   if (rows_staged)
@@ -180,7 +193,7 @@ __global__ void __launch_bounds__(kExpandThreads) k4_expand_direct(
         const int k = idx >> log2F;
         const u32 c = static_cast<u32>(idx) & fmask;
         const i64 par = row_of(max(s_rel[k], 0));
-        s_tq[idx] = static_cast<int>(dst_global(s_lo + k, par, c, 0));
+        s_tq[idx] = static_cast<int>(R[(rm.first + par) * F + c] + H[(s_lo + k - seg0) * F + c] - static_cast<u32>(s_rel[k]));
       }
       __syncthreads();
     }
