@@ -450,7 +450,7 @@ template <typename V, bool NUMERIC, int G, int LPN, int BT>
 static int launch_light_one(gm_plan* p, const int32_t* rows, const int* n_rows_dev, i64 n_rows_upper, int slots, int cap,
                             const i64* c_row_ptr, int32_t* c_col, V* c_val, i64 c_capacity, cudaStream_t st) {
   constexpr int kGroups = BT / G;
-  const size_t smem = kGroups * light_group_bytes<V, NUMERIC>(slots, cap);
+  const size_t smem = kGroups * light_group_bytes<V, NUMERIC>(slots, cap, G);
   auto kern = k3_light_rows<V, G, LPN, BT, NUMERIC>;
   // (static shared memory counts towards the 48 KB that need no opt-in)
   if (smem > 32 * 1024) GM_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)));

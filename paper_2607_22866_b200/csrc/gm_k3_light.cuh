@@ -39,11 +39,16 @@ __device__ __forceinline__ u32 hash_slot(int32_t col, u32 slots) {
 }
 
 // Shared-memory layout of one group: [sort buffer: cap x u64][values: slots x V][keys: slots x i32]
+// Groups narrower than a warp share one: their regions are staggered by `group` words, because power-of-two
+// region sizes would put the same array index of every group of a warp into the same bank (measured on the
+// 8-lane groups: half of all shared-memory wavefronts were conflict replays).
 template <typename V, bool NUMERIC>
-__host__ __device__ inline size_t light_group_bytes(int slots, int cap) {
+__host__ __device__ inline size_t light_group_bytes(int slots, int cap, int group) {
   size_t b = static_cast<size_t>(slots) * 4;
   if (NUMERIC) b += static_cast<size_t>(slots) * sizeof(V) + static_cast<size_t>(cap) * 8;
-  return (b + 15) & ~size_t{15};
+  b = (b + 15) & ~size_t{15};
+  if (group < 32) b += static_cast<size_t>(group) * 4;  // 8 lanes: 32 bytes, keeps 16-byte alignment
+  return b;
 }
 
 template <typename V, int G, int LPN, int BT, bool NUMERIC>
@@ -58,7 +63,7 @@ __global__ void __launch_bounds__(BT) k3_light_rows(
   constexpr int kGroups = BT / G;
   const int gid = threadIdx.x / G;   // group inside the block
   const int t = threadIdx.x % G;     // thread inside the group
-  unsigned char* base = smem_raw + static_cast<size_t>(gid) * light_group_bytes<V, NUMERIC>(slots, cap);
+  unsigned char* base = smem_raw + static_cast<size_t>(gid) * light_group_bytes<V, NUMERIC>(slots, cap, G);
   u64* sortbuf = reinterpret_cast<u64*>(base);
   V* vals = reinterpret_cast<V*>(base + (NUMERIC ? static_cast<size_t>(cap) * 8 : 0));
   int32_t* keys = reinterpret_cast<int32_t*>(base + (NUMERIC ? static_cast<size_t>(cap) * 8 + static_cast<size_t>(slots) * sizeof(V) : 0));
