@@ -377,6 +377,9 @@ def main():
     }
 
     if rank == 0 and not args.no_e2e:
+        # the host entry point uploads A and B itself: give it the whole device (no resident copies, no cached blocks)
+        del dA, dB
+        torch.cuda.empty_cache()
         try:
             line["e2e"] = e2e_leg(gm, torch, A, B, int(nnz), products, args.e2e_steps)
         except (gm.GmError, MemoryError, RuntimeError) as exc:  # the device-timed line above stands on its own
@@ -420,7 +423,7 @@ def e2e_leg(gm, torch, A, B, nnz, products, steps):
         avail = psutil.virtual_memory().available
     except Exception:
         avail = None
-    if avail is not None and need > 0.45 * avail:
+    if avail is not None and need > 0.7 * avail:
         return {"value": None, "unit": "GFLOP/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0,
                 "skipped": f"host buffers of {need / 1e9:.0f} GB for A, B and C do not fit beside the generator's "
                            f"copies in {avail / 1e9:.0f} GB of available host memory"}
