@@ -759,6 +759,7 @@ static int execute_t(gm_plan* p, cudaStream_t st, gm_csr* C) {
   int32_t* c_col = nullptr;
   V* c_val = nullptr;
   auto cleanup = [&]() {
+    if (p->sink && p->sink->copy_stream) cudaStreamSynchronize(p->sink->copy_stream);  // copies out of C in flight
     dev_free(c_row_ptr, st);
     dev_free(c_col, st);
     dev_free(c_val, st);
