@@ -368,9 +368,33 @@ static int build_plan(gm_plan* p, cudaStream_t st) {
                             cudaMemcpyDeviceToHost, st));
     GM_CUDA(cudaStreamSynchronize(st));
 
-    // ---- batches: consecutive heavy rows whose products fit one staging half-buffer
-    i64 stage = p->opts.stage_elems > 0 ? p->opts.stage_elems : (i64{1} << 29);
-    if (p->opts.stage_elems == 0) stage = std::max(stage, info.products_max_row);  // a row is never split
+    // The expansion writes the first level's children itself (see gm_k4_direct.cuh) unless asked to run that
+    // level as separate histogram and multisplit passes.
+    // That takes a row of F0 run starts per segment, which pays when segments are long compared with the
+    // fan-out (R-MAT products: ~1000 products per segment) and not when they are short (a clipped-Zipf pair
+    // with F0 = 256 and ~60 products per segment measured 3x slower that way).
+    const bool long_segments = prm.n_levels > 0 &&
+                               info.products_heavy >= 2 * static_cast<i64>(prm.fanout[0]) * std::max<i64>(info.nnz_a_heavy, 1);
+    // ... and a table of F0 + 1 boundaries per row of B, which must stay small (at most 1 GB, or what a staging
+    // buffer of the default size takes)
+    const i64 bound_bytes = prm.n_levels > 0 ? B.n_rows * static_cast<i64>(prm.fanout[0] + 1) * 4 : 0;
+    const bool bounds_fit = bound_bytes <= std::max<i64>(i64{1} << 30, std::min<i64>(info.products_heavy, i64{1} << 29) * (4 + p->sv));
+    p->direct = prm.n_levels > 0 && prm.fanout[0] <= 256 &&
+                (p->opts.level0_multisplit == 2 || (p->opts.level0_multisplit == 0 && long_segments && bounds_fit));
+    info.level0_direct = p->direct ? 1 : 0;
+    // one staging buffer is enough when no multisplit pass runs (no levels, or one level done by the expansion)
+    const int n_buf = prm.n_levels > (p->direct ? 1 : 0) ? 2 : 1;
+
+    // ---- batches: consecutive heavy rows whose products fit one staging buffer.  Default size: a fifth of the
+    // device's memory for staging (fewer, longer launches: on R-MAT scale 20, 2^31 products per batch instead of
+    // 2^29 took 7 % off the step), at least 2^29 products, at most what 32-bit tile positions allow.
+    i64 stage = p->opts.stage_elems;
+    if (stage <= 0) {
+      size_t free_b = 0, total_b = 0;
+      GM_CUDA(cudaMemGetInfo(&free_b, &total_b));
+      stage = std::max<i64>(i64{1} << 29, static_cast<i64>(total_b / 5) / (static_cast<i64>(n_buf) * (4 + p->sv)));
+      stage = std::max(stage, info.products_max_row);  // a row is never split
+    }
     stage = std::min(stage, info.products_heavy);
     const i64 kMaxStage = (i64{1} << 31) - kSplitTile;  // batch-relative positions are 32-bit in the multisplit tiles
     if (stage > kMaxStage) stage = kMaxStage;
@@ -386,7 +410,6 @@ static int build_plan(gm_plan* p, cudaStream_t st) {
     }
     // the accumulate kernel streams whole tiles: it may read (and ignore) up to one tile past the last product
     const size_t se = static_cast<size_t>(info.stage_elems) + 4096 + 8;
-    const int n_buf = prm.n_levels > 0 ? 2 : 1;
     for (int i = 0; i < n_buf; ++i) {
       GM_TRY(plan_alloc(p, &p->stage_col[i], se, st));
       unsigned char* v = nullptr;
@@ -408,18 +431,6 @@ static int build_plan(gm_plan* p, cudaStream_t st) {
     const size_t n_tiles_max = static_cast<size_t>(info.stage_elems) / std::min({kExpandTile, kSplitTile, kGatherTile}) + 2;
     GM_TRY(plan_alloc(p, &p->tile_meta, n_tiles_max, st));
     GM_TRY(plan_alloc(p, &p->row_meta, n_tiles_max, st));
-    // The expansion writes the first level's children itself (see gm_k4_direct.cuh) unless asked to run that
-    // level as separate histogram and multisplit passes.
-    // That takes a row of F0 run starts per segment, which pays when segments are long compared with the
-    // fan-out (R-MAT products: ~1000 products per segment) and not when they are short (a clipped-Zipf pair
-    // with F0 = 256 and ~60 products per segment measured 3x slower that way).
-    const bool long_segments = info.products_heavy >= 2 * static_cast<i64>(prm.fanout[0]) * std::max<i64>(info.nnz_a_heavy, 1);
-    // ... and a table of F0 + 1 boundaries per row of B, which must stay small next to the staging buffers
-    const i64 bound_bytes = B.n_rows * static_cast<i64>(prm.fanout[0] + 1) * 4;
-    const bool bounds_fit = bound_bytes <= std::max<i64>(i64{1} << 30, static_cast<i64>(se) * (4 + p->sv));
-    p->direct = prm.n_levels > 0 && prm.fanout[0] <= 256 &&
-                (p->opts.level0_multisplit == 2 || (p->opts.level0_multisplit == 0 && long_segments && bounds_fit));
-    info.level0_direct = p->direct ? 1 : 0;
     if (p->direct) {
       const int F0 = prm.fanout[0];
       i64 max_seg_b = 0;

@@ -273,10 +273,10 @@ def _check_sampled_rows(A, B, n_random=200, n_heavy=60, **opts):
 
 
 def test_config2_rmat20_full_size_sampled_rows():
-    # the benchmark's default workload: 2.1e10 products, 9.7e9 entries of C, dozens of batches
+    # the benchmark's default workload: 2.1e10 products, 9.7e9 entries of C, about ten batches of up to 2^31 products
     A, B, _ = gen.config_inputs(2)
     info, stats = _check_sampled_rows(A, B)
-    assert info.n_batches > 10 and info.params.levels() == [32] and stats.c_capacity >= stats.c_nnz
+    assert info.n_batches >= 8 and info.params.levels() == [32] and stats.c_capacity >= stats.c_nnz
 
 
 def test_config3_rmat_fp64_two_levels_sampled_rows():
