@@ -383,6 +383,7 @@ __global__ void __launch_bounds__(BT, 1) k6_accumulate(
         int spins = 0;
         while (!mbar_try_wait(&full_bar[st], par)) {
           __nanosleep(40);
+          if (*static_cast<volatile int*>(&s_abort)) break;  // somebody gave up: no tile will be issued any more
           if (++spins > kAccSpinLimit) { s_abort = 1; break; }
         }
         phase_bits ^= (1u << st);
@@ -534,12 +535,29 @@ __global__ void __launch_bounds__(BT, 1) k6_accumulate(
         ++kw;
         crow = (crow + 1u) & crow_mask;
       }
-      // ---- the stage is free again: refill it
-      __syncthreads();
-      if (s_abort) { aborted = true; break; }
-      if (tid == 0 && j + stages < n_tiles) issue(j + stages, st);
+      // ---- the stage is free again once every warp has finished the tile.  Only the warp that refills it has to
+      // wait for that: the others announce that they are done (named barrier 1 + stage) and go on to the next
+      // tile, whose data is in another stage.  A warp cannot arrive twice on a barrier before it has completed:
+      // its next use of this stage waits for the refill, which is issued after the barrier.
+      // (Only for the block that has an SM to itself: the named barriers of narrower blocks, several per SM, would
+      // not fit the SM's sixteen.)
+      if constexpr (BT == 1024) {
+        if (j + stages < n_tiles) {  // (uniform)
+          if (tid < 32) {
+            asm volatile("bar.sync %0, %1;" ::"r"(1 + st), "r"(BT) : "memory");
+            if (tid == 0 && !*static_cast<volatile int*>(&s_abort)) issue(j + stages, st);
+          } else {
+            asm volatile("bar.arrive %0, %1;" ::"r"(1 + st), "r"(BT) : "memory");
+          }
+        }
+      } else {
+        __syncthreads();
+        if (tid == 0 && j + stages < n_tiles && !*static_cast<volatile int*>(&s_abort)) issue(j + stages, st);
+      }
       st = (st + 1 == stages) ? 0 : st + 1;
     }
+    __syncthreads();  // every warp is through the segment
+    aborted = s_abort != 0;
     if (aborted) {
       // Tiles that were issued but not consumed still target this block's shared memory: give each a
       // bounded chance to land before the block exits (its barrier answers at once if it already did).
