@@ -533,14 +533,14 @@ static int launch_accumulate(gm_plan* p, const Batch& b, const HeavyBatchState<V
   const int ctas = prm.acc_ctas_per_sm;
   const size_t budget = p->smem_bytes / static_cast<size_t>(ctas) - 1024;
   const int bt = prm.acc_block_threads;
-  // four products per thread and tile when two such stages fit next to the accumulator (the per-tile control
-  // code is executed by every warp, so bigger tiles amortise it), otherwise two
-  int pt = 4;
-  int stages = acc_ring_stages(budget, W, sizeof(V), true, bt, pt);
-  if (stages < 2) {
-    pt = 2;
+  // the largest tile (four, three or two products per thread) of which two stages fit next to the accumulator:
+  // the per-tile control code is executed by every warp, so bigger tiles amortise it
+  int pt = 4, stages = 0;
+  for (; pt >= 2; --pt) {
     stages = acc_ring_stages(budget, W, sizeof(V), true, bt, pt);
+    if (stages >= 2) break;
   }
+  if (pt < 2) pt = 2;
   if (stages < 2) return fail(GM_ERR_UNSUPPORTED_SMEM, "shared memory budget too small for the accumulate kernel");
   const size_t smem = acc_stream_smem_bytes(W, sizeof(V), true, stages, bt, pt);
   const i64 n_segs = (b.elems + kAccSegment - 1) / kAccSegment;
@@ -572,7 +572,7 @@ static int launch_accumulate(gm_plan* p, const Batch& b, const HeavyBatchState<V
     kern<<<grid, BT, smem, st>>>(hs.fin_col, hs.fin_val, hs.chunk_off, hs.n_chunks, p->seg_first, n_segs, p->ticket, \
                                  hs.log2_cpr, W, stages, small_max, p->chunk_nnz, p->err);                                      \
   } while (0)
-#define GM_ACC(BT) do { if (pt == 4) GM_ACC2(BT, 4); else GM_ACC2(BT, 2); } while (0)
+#define GM_ACC(BT) do { if (pt == 4) GM_ACC2(BT, 4); else if (pt == 3) GM_ACC2(BT, 3); else GM_ACC2(BT, 2); } while (0)
   if (bt == 1024) GM_ACC(1024);
   else if (bt == 512) GM_ACC(512);
   else if (bt == 256) GM_ACC(256);
