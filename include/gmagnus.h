@@ -222,7 +222,9 @@ int gm_plan_get_row_products(const gm_plan* plan, int64_t* ip_out_device, void* 
  * Its scratch (products per stored entry, their prefix sums, tile sums of the scan) lives in a
  * fixed array inside the library image: about 12.6 MB of device memory on every GPU that loads the
  * library, held until the process exits.
- *   A, B           host structs with DEVICE pointers, as for gm_spgemm_plan (values are not read)
+ *   A, B           host structs with DEVICE pointers, as for gm_spgemm_plan; only row_ptr and col_idx are
+ *                  read, so vals may be NULL and dtype is ignored.  Columns of A are not range-checked:
+ *                  an entry of A.col_idx outside [0, B.n_rows) reads past B.row_ptr
  *   ip_out_device  DEVICE array of A->n_rows int64, written by the call
  *   cuda_stream    the work is enqueued there; the call does not synchronise
  * Limit: A->nnz <= GM_NOALLOC_MAX_NNZ_A (1,048,576); larger inputs are rejected with GM_ERR_CAPACITY

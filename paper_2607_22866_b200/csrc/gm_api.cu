@@ -214,13 +214,15 @@ static unsigned grid_for(i64 n, int threads, int num_sms, int per_sm = 16) {
   return static_cast<unsigned>(g);
 }
 
-static int check_csr_arg(const gm_csr* M, const char* name) {
+// structure_only: the caller reads row_ptr and col_idx alone (values and dtype are not looked at)
+static int check_csr_arg(const gm_csr* M, const char* name, bool structure_only = false) {
   if (!M) return fail(GM_ERR_INVALID_ARG, std::string(name) + " is null");
   if (M->n_rows < 0 || M->n_cols < 0 || M->nnz < 0 || M->n_cols > INT32_MAX || M->n_rows > INT32_MAX)
     return fail(GM_ERR_INVALID_ARG, std::string(name) + ": sizes out of range");
-  if (!M->row_ptr || (M->nnz > 0 && (!M->col_idx || !M->vals)))
+  if (!M->row_ptr || (M->nnz > 0 && (!M->col_idx || (!structure_only && !M->vals))))
     return fail(GM_ERR_INVALID_ARG, std::string(name) + ": null array");
-  if (M->dtype != GM_F32 && M->dtype != GM_F64) return fail(GM_ERR_DTYPE, std::string(name) + ": unknown dtype");
+  if (!structure_only && M->dtype != GM_F32 && M->dtype != GM_F64)
+    return fail(GM_ERR_DTYPE, std::string(name) + ": unknown dtype");
   return GM_OK;
 }
 
@@ -1168,14 +1170,6 @@ const char* gm_status_string(int status) {
 
 const char* gm_last_error(void) { return g_last_error.c_str(); }
 
-#ifdef GM_K6_PROFILE
-int gm_debug_k6_profile(unsigned long long* out16, int reset) {
-  cudaMemcpyFromSymbol(out16, g_k6_prof, 16 * sizeof(unsigned long long));
-  if (reset) { unsigned long long z[16] = {0}; cudaMemcpyToSymbol(g_k6_prof, z, sizeof(z)); }
-  return 0;
-}
-#endif
-
 }  // extern "C"
 
 // ------------------------------------------------------------------------------------------------
@@ -1208,8 +1202,8 @@ static int g_noalloc_sms[kNoAllocMaxDevices] = {0};
 }  // namespace gm
 
 extern "C" int gm_row_products_noalloc(const gm_csr* A, const gm_csr* B, int64_t* ip_out_device, void* cuda_stream) {
-  GM_TRY(check_csr_arg(A, "A"));
-  GM_TRY(check_csr_arg(B, "B"));
+  GM_TRY(check_csr_arg(A, "A", true));
+  GM_TRY(check_csr_arg(B, "B", true));
   if (!ip_out_device && A->n_rows > 0) return fail(GM_ERR_INVALID_ARG, "ip_out_device is null");
   if (A->n_cols != B->n_rows) return fail(GM_ERR_DIM_MISMATCH, "A.n_cols != B.n_rows");
   if (A->nnz > kNoAllocMaxNnz)

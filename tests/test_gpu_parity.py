@@ -246,7 +246,7 @@ def test_host_entry_point_streams_batches_to_the_host(dtype):
     assert ei.value.status == -6
 
 
-def _check_sampled_rows(A, B, n_random=200, n_heavy=60, **opts):
+def _check_sampled_rows(A, B, n_random=200, n_heavy=60, whole_row_ptr=False, **opts):
     """Full-size check in the launch configuration the benchmark times: structure and values of
     sampled rows (random rows, the heaviest rows, random heavy rows) against the row-range oracle,
     plus whole-matrix invariants that need no reference."""
@@ -257,6 +257,9 @@ def _check_sampled_rows(A, B, n_random=200, n_heavy=60, **opts):
     rp = C.row_ptr.cpu().numpy()
     assert rp[0] == 0 and rp[-1] == C.nnz == stats.c_nnz and np.all(np.diff(rp) >= 0)
     assert np.all(np.diff(rp) <= np.minimum(ip, B.n_cols)) and np.all((np.diff(rp) == 0) == (ip == 0))
+    if whole_row_ptr:
+        # every row's entry count against the oracle's count-only (symbolic) pass over the whole matrix
+        assert np.array_equal(np.diff(rp), oracle.spgemm_row_counts(A, B))
     rng = np.random.default_rng(0)
     rows = set(rng.integers(0, A.n_rows, n_random).tolist()) | set(np.argsort(-ip)[:3].tolist())
     heavy = np.nonzero(ip > info.params.tau)[0]
@@ -273,10 +276,28 @@ def _check_sampled_rows(A, B, n_random=200, n_heavy=60, **opts):
 
 
 def test_config2_rmat20_full_size_sampled_rows():
-    # the benchmark's default workload: 2.1e10 products, 9.7e9 entries of C, about ten batches of up to 2^31 products
+    # the benchmark's default workload: 2.1e10 products, 9.7e9 entries of C, about ten batches of up to 2^31 products;
+    # sampled rows in full, and the entry count of every row
     A, B, _ = gen.config_inputs(2)
-    info, stats = _check_sampled_rows(A, B)
+    info, stats = _check_sampled_rows(A, B, whole_row_ptr=True)
     assert info.n_batches >= 8 and info.params.levels() == [32] and stats.c_capacity >= stats.c_nnz
+    assert info.level0_direct == 1
+
+
+def test_config3_rmat21_fp64_full_size_default_plan():
+    # R-MAT scale 21, edge factor 8, fp64, exactly as the benchmark runs it (no plan options): one level of 128
+    # children written by the expansion kernel, several batches, a result of more than 100 GB
+    A, B, _ = gen.config_inputs(3)
+    info, stats = _check_sampled_rows(A, B, n_random=150, n_heavy=50)
+    assert info.params.levels() == [128] and info.level0_direct == 1 and info.n_batches > 1
+
+
+def test_config4_zipf_pair_full_size_default_plan():
+    # the rectangular clipped-Zipf pair (2^24 columns) exactly as the benchmark runs it: two levels, the first as
+    # separate passes (short segments) with its histogram counted by the expansion kernel, 256 children
+    A, B, _ = gen.config_inputs(4)
+    info, stats = _check_sampled_rows(A, B, n_random=150, n_heavy=60, whole_row_ptr=True)
+    assert info.params.levels() == [256, 2] and info.level0_direct == 0 and info.rows_heavy > 0
 
 
 def test_config3_rmat_fp64_two_levels_sampled_rows():
@@ -291,6 +312,17 @@ def test_config4_zipf_wide_columns_three_levels_sampled_rows():
     A, B, _ = gen.config_inputs(4, shrink=2)
     info, stats = _check_sampled_rows(A, B, n_random=60, n_heavy=40, max_fanout=8, chunk_width=8192)
     assert info.params.n_levels == 3 and info.rows_heavy > 0
+
+
+@pytest.mark.parametrize("separate", [0, 1])
+@pytest.mark.parametrize("dtype", [np.float32, np.float64])
+def test_first_level_of_256_children_as_separate_passes(dtype, separate):
+    # fan-out 256 with the first level run as histogram + multisplit passes over the staging buffer (the shape of the
+    # Zipf pair's default plan): rows of B are short, so the planner does not let the expansion place the products
+    A, B, _ = gen.config_inputs(4, shrink=5)
+    C, info, stats = check_product(A, B, tau=256, chunk_width=1024, separate_histogram=separate, stage_elems=1 << 18)
+    assert info.params.levels()[0] == 256 and info.params.n_levels == 2 and info.level0_direct == 0
+    assert info.n_batches > 1 and info.rows_heavy > 100
 
 
 @pytest.mark.parametrize("separate", [0, 1])

@@ -2,14 +2,15 @@
 budget, a latency-critical section, a host whose allocator belongs to another runtime):
 gm_row_products_noalloc computes the intermediate products per row with its scratch in a fixed array
 of the library image.  Checked here, through the C ABI, against the row analysis of gm_spgemm_plan
-(the existing entry point), bit for bit because the result is an integer count, on two calls in a
-row that share the scratch array.  This file sorts last so that a stop-at-first-failure run has
+(the existing entry point) and against the CPU oracle's count, bit for bit because the result is an
+integer count, on two calls in a row that share the scratch array.  This file sorts last so that a stop-at-first-failure run has
 already been through every other test."""
 import numpy as np
 import pytest
 import torch
 
 import gen
+import oracle
 
 pytestmark = pytest.mark.gpu
 
@@ -31,6 +32,9 @@ def test_no_alloc_row_products_matches_plan_twice_in_a_row():
     assert A1.nnz <= gm.NOALLOC_MAX_NNZ_A and A2.nnz <= gm.NOALLOC_MAX_NNZ_A
     cases = [(gm.DeviceCSR.from_host(A1),) * 2, (gm.DeviceCSR.from_host(A2), gm.DeviceCSR.from_host(B2))]
     refs = [_reference(gm, dA, dB) for dA, dB in cases]
+    # the plan's row analysis itself is pinned to the definition (CPU oracle), so both entry points are
+    for ref, (hA, hB) in zip(refs, [(A1, A1), (A2, B2)]):
+        assert np.array_equal(ref.cpu().numpy(), oracle.row_products(hA, hB))
     outs = [torch.full((dA.n_rows,), -7, dtype=torch.int64, device="cuda") for dA, _ in cases]
     torch.cuda.synchronize()
     before = torch.cuda.memory_allocated()
@@ -38,8 +42,9 @@ def test_no_alloc_row_products_matches_plan_twice_in_a_row():
         gm.row_products_noalloc(dA, dB, out)
     assert torch.cuda.memory_allocated() == before   # nothing came from torch's allocator (the library's hook)
     torch.cuda.synchronize()
-    for out, ref in zip(outs, refs):
+    for out, ref, (hA, hB) in zip(outs, refs, [(A1, A1), (A2, B2)]):
         assert torch.equal(out, ref)
+        assert np.array_equal(out.cpu().numpy(), oracle.row_products(hA, hB))
     # and once more in the other order: the scratch is reused, nothing needs clearing
     for (dA, dB), out, ref in reversed(list(zip(cases, outs, refs))):
         out.fill_(-1)
