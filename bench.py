@@ -198,6 +198,7 @@ def kernel_table(info, stats_avg, sv, nnz_b, n_light_entries_a):
     nnz_c, nnz_ch = stats_avg["c_nnz"], stats_avg["c_nnz_heavy"]
     chunks = stats_avg["final_chunks"]
     e_small, nnz_small = stats_avg["small_chunk_products"], stats_avg["small_chunk_entries"]
+    e_mid, nnz_mid = stats_avg["mid_chunk_products"], stats_avg["mid_chunk_entries"]
     parents = [rows_h]
     for l in range(L):
         parents.append(parents[-1] * p.fanout[l])
@@ -214,9 +215,12 @@ def kernel_table(info, stats_avg, sv, nnz_b, n_light_entries_a):
                       stats_avg["ms_expand"]),
         "k5a_histogram": (hist + seg_tables, stats_avg["ms_histogram"]),
         "k5b_multisplit": (split, stats_avg["ms_multisplit"]),
-        # chunks of few products are sorted by one warp each; the streaming kernel owes the rest
+        # chunks of few products are sorted by one warp each, mid-size ones take a small block each (its second pass
+        # re-reads the chunk from L2: not counted), the dense-accumulator kernel owes the rest
         "k6_small_chunks": (se * e_small + se * nnz_small + 12 * chunks, stats_avg["ms_small_chunks"]),
-        "k6_accumulate": (se * (e - e_small) + se * (nnz_ch - nnz_small) + 12 * chunks, stats_avg["ms_accumulate"]),
+        "k6_mid_chunks": (se * e_mid + se * nnz_mid, stats_avg["ms_mid_chunks"]),
+        "k6_accumulate": (se * (e - e_small - e_mid) + se * (nnz_ch - nnz_small - nnz_mid) + 12 * chunks,
+                          stats_avg["ms_accumulate"]),
         "k7_gather": (2 * se * nnz_ch + 24 * chunks, stats_avg["ms_gather"]),
     }
     return {k: {"bytes": int(b), "ms": float(ms), "gbs": (b / ms / 1e6 if ms > 0 else 0.0)} for k, (b, ms) in tbl.items()}
@@ -353,7 +357,7 @@ def main():
     n_split = max(info.params.n_levels - (1 if info.level0_direct else 0), 1)
     per_launch = {"k4_expand": n_b, "k5a_histogram": n_b * n_split,
                   "k5b_multisplit": n_b * n_split, "k6_accumulate": n_b,
-                  "k6_small_chunks": n_b, "k7_gather": n_b}.get(dom, 1)
+                  "k6_small_chunks": n_b, "k6_mid_chunks": n_b, "k7_gather": n_b}.get(dom, 1)
     roofline = {"kernel": dom, "bound": "hbm", "achieved": kt[dom]["gbs"], "peak": peak, "unit": "GB/s",
                 "frac": kt[dom]["gbs"] / peak, "peak_kind": f"of {peak_kind}",
                 "traffic": (kt[dom]["bytes"] / per_launch * TRAFFIC_RATIO[dom]) if dom in TRAFFIC_RATIO else None,

@@ -79,7 +79,13 @@ typedef struct gm_plan_opts {
                               the staging buffer (Algorithm 5 as printed); 2 = the expansion kernel writes
                               the first level's children itself; 0 (default) = the latter when the heavy
                               rows' segments are long compared with the fan-out, else the former        */
-  int32_t reserved[6];
+  int32_t small_chunk_max; /* final chunks of at most this many products are sorted by one warp each (Section
+                              III-A's branch for light chunks); 0 = default (512), -1 = none, at most 512        */
+  int32_t mid_chunk_max;   /* final chunks of at most this many products (and more than small_chunk_max) get one
+                              128-thread block each, symbolic then numeric pass over a compact array; larger
+                              ones go to the dense W-column accumulator.  0 = default (4096 for fp32, 2048 for
+                              fp64, less when shared memory is short), -1 = none                                 */
+  int32_t reserved[4];
 } gm_plan_opts;
 
 /* What the host planner derives from (C.m, value size, smem_bytes): Section III-D. */
@@ -127,8 +133,11 @@ typedef struct gm_exec_stats {
   int64_t small_chunk_entries;  /* entries of C those chunks produced                            */
   float ms_light_symbolic, ms_light_numeric, ms_expand, ms_histogram, ms_multisplit,
       ms_accumulate, ms_gather, ms_scan, ms_total;
-  float ms_small_chunks;       /* the one-warp-per-chunk kernel; ms_accumulate is the streaming kernel alone */
-  float reserved[4];
+  float ms_small_chunks;       /* the one-warp-per-chunk kernel; ms_accumulate is the dense-accumulator kernel alone */
+  float ms_mid_chunks;         /* the one-small-block-per-chunk kernel                                          */
+  float reserved[3];
+  int64_t mid_chunk_products;  /* products in chunks handled by the one-small-block-per-chunk kernel             */
+  int64_t mid_chunk_entries;   /* entries of C those chunks produced                                             */
 } gm_exec_stats;
 
 typedef struct gm_plan gm_plan; /* opaque, owned by the library */
@@ -177,8 +186,9 @@ int gm_spgemm_plan_ex(const gm_csr* A, const gm_csr* B, size_t smem_bytes,
  * (symbolic, then numeric); heavy rows, batch by batch, through the expansion (outer-product)
  * kernel (Algorithm 4), one histogram + multisplit (Algorithm 5) per level (by default the first
  * level is done by the expansion kernel itself, see gm_plan_opts.level0_multisplit), the
- * chunk-accumulate kernels (small chunks by a one-warp sort, the others in the dense shared-memory
- * accumulator of Section III-E; every chunk is compacted in place and its entries counted) and, once
+ * chunk-accumulate kernels (the chunks are binned by size as in Section III-E: small ones by a one-warp
+ * sort, mid-size ones by a small block in a symbolic and a numeric pass, the others in the dense
+ * shared-memory accumulator; every chunk is compacted in place and its entries counted) and, once
  * C.row_ptr is known by prefix sums over the per-row counts, the gather of the chunks into C.
  *   C_out  host struct filled with device pointers allocated through the allocator hook;
  *          C_out->nnz is exact.  Release with gm_csr_free.

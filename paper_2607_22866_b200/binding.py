@@ -43,7 +43,8 @@ class PlanOpts(ctypes.Structure):
                 ("acc_ctas_per_sm", ctypes.c_int32), ("stage_elems", ctypes.c_int64),
                 ("c_capacity", ctypes.c_int64), ("separate_histogram", ctypes.c_int32),
                 ("validate_inputs", ctypes.c_int32), ("single_stream", ctypes.c_int32),
-                ("level0_multisplit", ctypes.c_int32), ("reserved", ctypes.c_int32 * 6)]
+                ("level0_multisplit", ctypes.c_int32), ("small_chunk_max", ctypes.c_int32),
+                ("mid_chunk_max", ctypes.c_int32), ("reserved", ctypes.c_int32 * 4)]
 
 
 class Params(ctypes.Structure):
@@ -73,7 +74,8 @@ class ExecStats(ctypes.Structure):
                 ("ms_light_symbolic", ctypes.c_float), ("ms_light_numeric", ctypes.c_float),
                 ("ms_expand", ctypes.c_float), ("ms_histogram", ctypes.c_float), ("ms_multisplit", ctypes.c_float),
                 ("ms_accumulate", ctypes.c_float), ("ms_gather", ctypes.c_float), ("ms_scan", ctypes.c_float),
-                ("ms_total", ctypes.c_float), ("ms_small_chunks", ctypes.c_float), ("reserved", ctypes.c_float * 4)]
+                ("ms_total", ctypes.c_float), ("ms_small_chunks", ctypes.c_float), ("ms_mid_chunks", ctypes.c_float),
+                ("reserved", ctypes.c_float * 3), ("mid_chunk_products", ctypes.c_int64), ("mid_chunk_entries", ctypes.c_int64)]
 
 
 _ALLOC_FN = ctypes.CFUNCTYPE(ctypes.c_void_p, ctypes.c_size_t, ctypes.c_void_p, ctypes.c_void_p)

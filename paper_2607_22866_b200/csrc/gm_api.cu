@@ -93,7 +93,7 @@ struct Buf {
 // plan
 // ------------------------------------------------------------------------------------------------
 struct PhaseTimes {
-  enum Phase { kLightSym, kLightNum, kExpand, kHist, kSplit, kAccSym, kAccNum, kAccSmall, kScan, kCount };
+  enum Phase { kLightSym, kLightNum, kExpand, kHist, kSplit, kAccSym, kAccNum, kAccSmall, kAccMid, kScan, kCount };
   struct Rec { int phase; cudaEvent_t a, b; };
   std::vector<Rec> recs;
   std::vector<cudaEvent_t> pool;
@@ -165,6 +165,7 @@ struct gm_plan {
   uint32_t* seg_h = nullptr;       // H: segments of a batch x F0 (G minus the child boundary of the segment's row of B)
   uint32_t* seg_tile_sums = nullptr;
   bool direct = false;             // the expansion writes the level-0 children itself
+  int small_max = 0, mid_max = 0;  // size classes of the final chunks: <= small_max one warp, <= mid_max one small block
   std::vector<int64_t> heavy_nz_off_host;
   int64_t* heavy_nz_off = nullptr; // nH + 1
   int32_t* sym_rows = nullptr;     // bins x nA
@@ -173,7 +174,8 @@ struct gm_plan {
   int* num_fill = nullptr;         // 8
   int32_t* row_nnz = nullptr;      // nA
   int64_t* scan_tmp = nullptr;
-  int64_t* c_total = nullptr;      // [0] running nnz(C) (device carry), [1] heavy entries, [2] products and [3] entries of small chunks
+  int64_t* c_total = nullptr;      // [0] running nnz(C) (device carry), [1] heavy entries, [2] products and [3] entries of
+                                   // small chunks, [4] products and [5] entries of mid-size chunks
   int* err = nullptr;
   // heavy workspace
   int32_t* stage_col[2]{};
@@ -184,8 +186,9 @@ struct gm_plan {
   gm::u32* chunk_nnz = nullptr;
   int64_t* chunk_nnz_off = nullptr;
   int64_t* chunk_base = nullptr;   // numeric pass: position in C of every chunk's first entry
-  int64_t* seg_first = nullptr;    // accumulate kernel: first chunk of every element segment
-  int* ticket = nullptr;
+  int32_t* mid_list = nullptr;     // accumulate kernels: chunks of the mid-size class
+  int32_t* big_list = nullptr;     // ... and of the big class (the longest from the front, the others from the back)
+  int* acc_counters = nullptr;     // list lengths and tickets (see k6_classify)
   gm::TileMeta* row_meta = nullptr;   // per tile of the expansion kernel: heavy rows it touches (fused histogram)
   gm::TileMeta* tile_meta = nullptr;  // per tile of the expansion / multisplit kernels: groups it touches
   gm::PhaseTimes times;
@@ -261,6 +264,17 @@ static int build_plan(gm_plan* p, cudaStream_t st) {
     if (rc != GM_OK) return fail(rc, "planner rejected the parameters");
   }
   const gm_params& prm = info.params;
+  {
+    // size classes of the final chunks (Section III-E bins chunks by size)
+    const gm_plan_opts& o = p->opts;
+    if (o.small_chunk_max < -1 || o.small_chunk_max > kAccSmallChunk || o.mid_chunk_max < -1 || o.mid_chunk_max > (1 << 15))
+      return fail(GM_ERR_INVALID_ARG, "small_chunk_max / mid_chunk_max out of range");
+    p->small_max = o.small_chunk_max < 0 ? 0 : (o.small_chunk_max ? o.small_chunk_max : kAccSmallChunk);
+    int mid = o.mid_chunk_max < 0 ? 0 : (o.mid_chunk_max ? o.mid_chunk_max : (p->sv == 4 ? 4096 : 2048));
+    // several mid-chunk blocks must fit an SM next to each other for the class to pay
+    while (mid > p->small_max && mid_smem_bytes(prm.chunk_width, p->sv, mid) + 1024 > p->smem_bytes / 8) mid /= 2;
+    p->mid_max = std::max(mid, p->small_max);
+  }
 
   GM_TRY(plan_alloc(p, &p->err, 4, st));
   GM_CUDA(cudaMemsetAsync(p->err, 0, 4 * sizeof(int), st));
@@ -288,7 +302,7 @@ static int build_plan(gm_plan* p, cudaStream_t st) {
   GM_TRY(plan_alloc(p, &heavy_pos, static_cast<size_t>(nA) + 1, st));
   GM_TRY(plan_alloc(p, &totals, 1, st));
   GM_TRY(plan_alloc(p, &p->row_nnz, static_cast<size_t>(nA) + 1, st));
-  GM_TRY(plan_alloc(p, &p->c_total, 4, st));
+  GM_TRY(plan_alloc(p, &p->c_total, 8, st));
   GM_TRY(plan_alloc(p, &p->scan_tmp, static_cast<size_t>(scan_tmp_elems(std::max<i64>(std::max(nnzA, nA), 1))), st));
   GM_CUDA(cudaMemsetAsync(totals, 0, sizeof(K1Totals), st));
   if (nnzA > 0) k1_nz_len<<<grid_for(nnzA, 256, p->num_sms, 32), 256, 0, st>>>(A.col_idx, nnzA, B.row_ptr, nz_len);
@@ -428,8 +442,9 @@ static int build_plan(gm_plan* p, cudaStream_t st) {
     GM_TRY(plan_alloc(p, &p->chunk_nnz, n_chunks_max + 1, st));
     GM_TRY(plan_alloc(p, &p->chunk_nnz_off, n_chunks_max + 1, st));
     GM_TRY(plan_alloc(p, &p->chunk_base, n_chunks_max + 1, st));
-    GM_TRY(plan_alloc(p, &p->seg_first, static_cast<size_t>(info.stage_elems / kAccSegment) + 4, st));
-    GM_TRY(plan_alloc(p, &p->ticket, 4, st));
+    GM_TRY(plan_alloc(p, &p->mid_list, n_chunks_max + 1, st));
+    GM_TRY(plan_alloc(p, &p->big_list, n_chunks_max + 1, st));
+    GM_TRY(plan_alloc(p, &p->acc_counters, 8, st));
     const size_t n_tiles_max = static_cast<size_t>(info.stage_elems) / std::min({kExpandTile, kSplitTile, kGatherTile}) + 2;
     GM_TRY(plan_alloc(p, &p->tile_meta, n_tiles_max, st));
     GM_TRY(plan_alloc(p, &p->row_meta, n_tiles_max, st));
@@ -528,34 +543,18 @@ struct HeavyBatchState {
 };
 
 // K6: accumulate every chunk of the batch and compact it in place; chunk_nnz receives the entry counts.
+// Three kernels, one per size class of the chunks (see gm_k6_accumulate.cuh).
 template <typename V>
 static int launch_accumulate(gm_plan* p, const Batch& b, const HeavyBatchState<V>& hs, cudaStream_t st) {
   const gm_params& prm = p->info.params;
   const int W = prm.chunk_width;
-  const int ctas = prm.acc_ctas_per_sm;
-  const size_t budget = p->smem_bytes / static_cast<size_t>(ctas) - 1024;
   const int bt = prm.acc_block_threads;
-  // the largest tile (four, three or two products per thread) of which two stages fit next to the accumulator:
-  // the per-tile control code is executed by every warp, so bigger tiles amortise it
-  int pt = 4, stages = 0;
-  for (; pt >= 2; --pt) {
-    stages = acc_ring_stages(budget, W, sizeof(V), true, bt, pt);
-    if (stages >= 2) break;
-  }
-  if (pt < 2) pt = 2;
-  if (stages < 2) return fail(GM_ERR_UNSUPPORTED_SMEM, "shared memory budget too small for the accumulate kernel");
-  const size_t smem = acc_stream_smem_bytes(W, sizeof(V), true, stages, bt, pt);
-  const i64 n_segs = (b.elems + kAccSegment - 1) / kAccSegment;
-  k6_prepare<<<static_cast<unsigned>((n_segs + 1 + 255) / 256), 256, 0, st>>>(hs.chunk_off, hs.n_chunks, n_segs, p->seg_first);
-  GM_CUDA(cudaMemsetAsync(p->ticket, 0, sizeof(int), st));
+  const int small_max = p->small_max, mid_max = p->mid_max;
+  GM_CUDA(cudaMemsetAsync(p->acc_counters, 0, 8 * sizeof(int), st));
   GM_CUDA(cudaMemsetAsync(p->chunk_nnz, 0, static_cast<size_t>(hs.n_chunks) * sizeof(u32), st));
-  const int per_sm = 1024 / bt;
-  // chunks of at most small_max products go to the warp-per-chunk kernel (GM_SMALL_CHUNK=0 sends all of them
-  // through the block-wide accumulator: a debugging aid)
-  static const int small_max = [] {
-    const char* e = std::getenv("GM_SMALL_CHUNK");
-    return e ? std::max(0, std::min(std::atoi(e), kAccSmallChunk)) : kAccSmallChunk;
-  }();
+  k6_classify<<<grid_for(hs.n_chunks, 256, p->num_sms), 256, 0, st>>>(hs.chunk_off, hs.n_chunks, small_max, mid_max, p->mid_list,
+                                                                     p->big_list, p->acc_counters);
+  ++p->stats.launches;
   if (small_max > 0) {
     p->times.begin(PhaseTimes::kAccSmall, st);
     k6_small_chunks<V><<<static_cast<unsigned>(p->num_sms * 8), kSmallWarps * 32, 0, st>>>(
@@ -564,25 +563,39 @@ static int launch_accumulate(gm_plan* p, const Batch& b, const HeavyBatchState<V
     ++p->stats.launches;
     p->times.end(st);
   }
+  if (mid_max > small_max) {
+    p->times.begin(PhaseTimes::kAccMid, st);
+    const size_t smem = mid_smem_bytes(W, sizeof(V), mid_max);
+    auto kern = k6_mid_chunks<V>;
+    if (smem > 32 * 1024) GM_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)));
+    const int per_sm = std::max<int>(1, std::min<int>(2048 / kMidThreads, static_cast<int>((p->smem_bytes - 1024) / (smem + 1024))));
+    const unsigned grid = static_cast<unsigned>(std::min<i64>(hs.n_chunks, static_cast<i64>(p->num_sms) * per_sm));
+    kern<<<grid, kMidThreads, smem, st>>>(hs.fin_col, hs.fin_val, hs.chunk_off, p->mid_list, p->acc_counters, hs.log2_cpr, W,
+                                          mid_max, p->chunk_nnz, reinterpret_cast<u64*>(p->c_total + 4));
+    ++p->stats.launches;
+    p->times.end(st);
+  }
   p->times.begin(PhaseTimes::kAccNum, st);
-  const unsigned grid = static_cast<unsigned>(std::min<i64>(n_segs, static_cast<i64>(p->num_sms) * per_sm));
-#define GM_ACC2(BT, PT)                                                                                              \
+  {
+    const size_t smem = acc_smem_bytes_big(W, sizeof(V));
+    const int per_sm = 1024 / bt;
+    const unsigned grid = static_cast<unsigned>(std::min<i64>(hs.n_chunks, static_cast<i64>(p->num_sms) * per_sm));
+#define GM_ACC(BT)                                                                                                   \
   do {                                                                                                               \
-    auto kern = k6_accumulate<V, true, BT, PT>;                                                                      \
+    auto kern = k6_accumulate<V, BT>;                                                                                \
     if (smem > 32 * 1024)                                                                                            \
       GM_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)));     \
-    kern<<<grid, BT, smem, st>>>(hs.fin_col, hs.fin_val, hs.chunk_off, hs.n_chunks, p->seg_first, n_segs, p->ticket, \
-                                 hs.log2_cpr, W, stages, small_max, p->chunk_nnz, p->err);                                      \
+    kern<<<grid, BT, smem, st>>>(hs.fin_col, hs.fin_val, hs.chunk_off, hs.n_chunks, p->big_list, p->acc_counters,    \
+                                 hs.log2_cpr, W, p->chunk_nnz);                                                      \
   } while (0)
-#define GM_ACC(BT) do { if (pt == 4) GM_ACC2(BT, 4); else if (pt == 3) GM_ACC2(BT, 3); else GM_ACC2(BT, 2); } while (0)
-  if (bt == 1024) GM_ACC(1024);
-  else if (bt == 512) GM_ACC(512);
-  else if (bt == 256) GM_ACC(256);
-  else GM_ACC(128);
+    if (bt == 1024) GM_ACC(1024);
+    else if (bt == 512) GM_ACC(512);
+    else if (bt == 256) GM_ACC(256);
+    else GM_ACC(128);
 #undef GM_ACC
-#undef GM_ACC2
+  }
   p->times.end(st);
-  p->stats.launches += 2;
+  ++p->stats.launches;
   GM_CUDA(cudaGetLastError());
   return GM_OK;
 }
@@ -764,7 +777,7 @@ static int execute_t(gm_plan* p, cudaStream_t st, gm_csr* C) {
 
   GM_CUDA(cudaMemsetAsync(p->err, 0, sizeof(int), st));
   GM_CUDA(cudaMemsetAsync(p->row_nnz, 0, static_cast<size_t>(nA + 1) * sizeof(int32_t), st));
-  GM_CUDA(cudaMemsetAsync(p->c_total, 0, 4 * sizeof(int64_t), st));
+  GM_CUDA(cudaMemsetAsync(p->c_total, 0, 8 * sizeof(int64_t), st));
 
   // ---- result row_ptr
   i64* c_row_ptr = static_cast<i64*>(dev_alloc(static_cast<size_t>(nA + 1) * sizeof(i64), st));
@@ -851,7 +864,7 @@ static int execute_t(gm_plan* p, cudaStream_t st, gm_csr* C) {
       const i64 hi = std::max<i64>(1, std::min<i64>(info.c_nnz_upper, std::max(by_total, by_free)));
       const i64 lo = std::max<i64>(1, std::min<i64>(info.c_nnz_upper, by_free));
       tries.push_back(hi);
-      for (int k = 1; k <= 3 && hi > lo; ++k) tries.push_back(hi - (hi - lo) * k / 3);
+      for (int k = 1; k <= 8 && hi > lo; ++k) tries.push_back(hi - (hi - lo) * k / 8);
     }
     for (i64 cand : tries) {
       capacity = cand;
@@ -911,8 +924,8 @@ static int execute_t(gm_plan* p, cudaStream_t st, gm_csr* C) {
     }
   }
   if (tm.enabled) cudaEventRecord(ev_total1, st);
-  i64 tail_totals[3] = {0, 0, 0};  // heavy entries, small-chunk products, small-chunk entries
-  cudaMemcpyAsync(tail_totals, p->c_total + 1, 3 * sizeof(i64), cudaMemcpyDeviceToHost, st);
+  i64 tail_totals[5] = {0, 0, 0, 0, 0};  // heavy entries; products and entries of small chunks; of mid-size chunks
+  cudaMemcpyAsync(tail_totals, p->c_total + 1, 5 * sizeof(i64), cudaMemcpyDeviceToHost, st);
   cudaError_t e1 = cudaMemcpyAsync(&dev_err, p->err, sizeof(int), cudaMemcpyDeviceToHost, st);
   cudaError_t e2 = cudaStreamSynchronize(st);
   if (e1 != cudaSuccess || e2 != cudaSuccess) {
@@ -930,6 +943,8 @@ static int execute_t(gm_plan* p, cudaStream_t st, gm_csr* C) {
   p->stats.c_nnz_heavy = heavy_total;
   p->stats.small_chunk_products = tail_totals[1];
   p->stats.small_chunk_entries = tail_totals[2];
+  p->stats.mid_chunk_products = tail_totals[3];
+  p->stats.mid_chunk_entries = tail_totals[4];
   p->stats.c_capacity = capacity;
   if (tm.enabled) {
     float ph[PhaseTimes::kCount];
@@ -942,6 +957,7 @@ static int execute_t(gm_plan* p, cudaStream_t st, gm_csr* C) {
     p->stats.ms_gather = ph[PhaseTimes::kAccSym];
     p->stats.ms_accumulate = ph[PhaseTimes::kAccNum];
     p->stats.ms_small_chunks = ph[PhaseTimes::kAccSmall];
+    p->stats.ms_mid_chunks = ph[PhaseTimes::kAccMid];
     p->stats.ms_scan = ph[PhaseTimes::kScan];
     cudaEventElapsedTime(&p->stats.ms_total, ev_total0, ev_total1);
   }

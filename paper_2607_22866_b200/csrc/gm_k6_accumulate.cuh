@@ -1,86 +1,69 @@
 // K6 — chunk accumulation (the dense accumulator of Section III-E applied to the rows of
 // C^_reord): every final chunk (heavy row h, chunk c) owns the W consecutive columns
-// [c*W, (c+1)*W), so its products are summed into a W-entry dense accumulator in shared memory; a
-// bitmap records which columns received a product (structural zeros are kept), a block-wide prefix
-// sum over the bitmap words gives every occupied column its rank, and the chunk is written to C in
-// ascending column order.
+// [c*W, (c+1)*W), so its products can be summed in shared memory; a bitmap records which columns
+// received a product (structural zeros are kept), a prefix sum over the bitmap words gives every
+// occupied column its rank, and the chunk comes out in ascending column order.
 //
-// One pass, no symbolic twin: the position of a chunk in C is only known once every earlier chunk has been
-// counted, so the kernel writes the compacted chunk *in place*, over the start of the chunk's own (already
-// consumed) products in the staging buffer — the output of a chunk never has more entries than its input —
-// and reports the entry count.  A prefix sum over those counts gives C.rowPtr, and the gather kernel below
-// moves the compacted chunks to   C.rowPtr[row] + (entries of the row's earlier chunks).
+// One pass over the staging buffer, no symbolic twin: the position of a chunk in C is only known once
+// every earlier chunk has been counted, so each kernel writes the compacted chunk *in place*, over the
+// start of the chunk's own (already consumed) products — the output of a chunk never has more entries
+// than its input — and reports the entry count.  A prefix sum over those counts gives C.rowPtr, and the
+// gather kernel moves the compacted chunks to  C.rowPtr[row] + (entries of the row's earlier chunks).
 //
-// B200 design.  The chunks of a batch lie back to back in the staging buffer, so the kernel does
-// not fetch chunk by chunk: the element space is cut into equal segments (static flattened
-// partition, as in Algorithms 4 and 5), persistent blocks claim segments with a ticket, and each
-// block *streams* its segment through a ring of shared-memory tiles filled by bulk asynchronous
-// copies (cp.async.bulk + mbarrier), independent of chunk boundaries.  A chunk boundary only
-// triggers a flush of the accumulator.  The flush cleans what it writes, so a chunk costs time
-// proportional to its products and its output, not to W.  All waits are bounded.
+// B200 design.  The chunks of a power-law product span five orders of magnitude (most hold a few dozen
+// products, a few hold millions), and what a chunk costs beyond its products is the width of the team
+// that has to synchronise for it.  So the chunks are binned by size (the binning of Section III-E) and
+// every bin gets a team of its own width:
+//   k6_classify      one thread per chunk: lists of the mid-size and of the big chunks
+//   k6_small_chunks  n <= 512 products: one warp per chunk, register sort, no barrier at all
+//   k6_mid_chunks    n <= a few thousand: one 128-thread block per chunk, several blocks per SM.  Symbolic
+//                    then numeric as in Algorithm 3: pass 1 sets the column bitmap, a prefix sum over the
+//                    bitmap words ranks the columns, pass 2 adds every product to a *compact* array of the
+//                    chunk's entries (its size is bounded by the chunk's products, not by W, which is what
+//                    lets many chunks share an SM); the second pass re-reads the chunk from L2
+//   k6_accumulate    the rest: one 1024-thread block per SM with the dense W-column accumulator, products
+//                    streamed from HBM with 16-byte loads one tile ahead in registers, one flush per chunk
+// All of them are persistent grids that take chunks from a list with an atomic ticket; nothing waits on
+// anything but block-wide barriers.
 #pragma once
 #include "gm_common.cuh"
 
 namespace gm {
 
-// A block of BT threads streams tiles of PT * BT products (PT = 2 or 4 per thread) and keeps the offsets of BT
-// chunks at a time in shared memory.  Few threads with several products each: the per-tile and per-chunk
-// control code is executed by every warp, so a wide block multiplies it.
-constexpr i64 kAccSegment = i64{1} << 18;  // elements per ticket
-constexpr int kAccSpinLimit = 1 << 24;  // polls of an mbarrier before the kernel gives up
+constexpr int kMidThreads = 128;        // threads of one mid-chunk team
+constexpr int kHugeChunk = 1 << 16;     // big chunks with more products than this are handed out first
 
-__device__ __forceinline__ u32 smem_u32(const void* p) { return static_cast<u32>(__cvta_generic_to_shared(p)); }
-
-__device__ __forceinline__ void mbar_init(u64* bar, int count) {
-  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count) : "memory");
-}
-__device__ __forceinline__ void mbar_expect_tx(u64* bar, u32 bytes) {
-  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ bool mbar_try_wait(u64* bar, u32 parity) {
-  u32 ok;
-  asm volatile(
-      "{\n\t.reg .pred p;\n\t"
-      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-      "selp.u32 %0, 1, 0, p;\n\t}"
-      : "=r"(ok)
-      : "r"(smem_u32(bar)), "r"(parity)
-      : "memory");
-  return ok != 0;
-}
-// 1-D bulk copy global -> this block's shared memory; both addresses 16-byte aligned, bytes a multiple of 16
-__device__ __forceinline__ void bulk_g2s(void* dst, const void* src, u32 bytes, u64* bar) {
-  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(smem_u32(dst)),
-               "l"(src), "r"(bytes), "r"(smem_u32(bar))
-               : "memory");
-}
-
-// Number of ring stages that fit next to the accumulator of a block of `bt` threads.
-__host__ __device__ inline int acc_ring_stages(size_t smem_budget, int W, int val_bytes, bool numeric, int bt, int pt) {
-  const size_t fixed = static_cast<size_t>(W / 32) * 12 + (numeric ? static_cast<size_t>(W) * val_bytes : 0) +
-                       static_cast<size_t>(bt) * 4 + 256;
-  const size_t stage = static_cast<size_t>(pt * bt) * (4 + (numeric ? val_bytes : 0));
-  if (smem_budget <= fixed) return 0;
-  size_t s = (smem_budget - fixed) / stage;
-  return static_cast<int>(s > 8 ? 8 : s);
-}
-__host__ __device__ inline size_t acc_stream_smem_bytes(int W, int val_bytes, bool numeric, int stages, int bt, int pt) {
-  return static_cast<size_t>(W / 32) * 12 + (numeric ? static_cast<size_t>(W) * val_bytes : 0) +
-         static_cast<size_t>(bt) * 4 +
-         static_cast<size_t>(stages) * pt * bt * (4 + (numeric ? val_bytes : 0)) + 256;
-}
-
-// seg_first[s] = first chunk whose start offset is >= s * kAccSegment (s = 0..n_segs).
-__global__ void k6_prepare(const i64* __restrict__ chunk_off, i64 n_chunks, i64 n_segs, i64* __restrict__ seg_first) {
-  const i64 i = static_cast<i64>(blockIdx.x) * blockDim.x + threadIdx.x;
-  if (i <= n_segs) {
-    const i64 target = i * kAccSegment;
-    i64 lo = 0, hi = n_chunks;  // first k in [0, n_chunks] with chunk_off[k] >= target
-    while (lo < hi) {
-      const i64 mid = (lo + hi) >> 1;
-      if (chunk_off[mid] >= target) hi = mid; else lo = mid + 1;
+// Lists for the mid and big kernels.  Chunk ids are batch-relative and fit 32 bits.  Big chunks above kHugeChunk
+// are appended from the front of big_list, the others from its back, so that a ticket order front-to-back gives
+// the long ones out first (fewer blocks idle at the end of the launch).
+// counters: [0] mid chunks, [1] huge chunks, [2] other big chunks, [3] ticket of the mid kernel, [4] ticket of
+// the big kernel (all zeroed by the host before the launch).
+__global__ void k6_classify(const i64* __restrict__ chunk_off, i64 n_chunks, int small_max, int mid_max,
+                            int32_t* __restrict__ mid_list, int32_t* __restrict__ big_list, int* __restrict__ counters) {
+  const int lane = threadIdx.x & 31;
+  for (i64 k0 = (static_cast<i64>(blockIdx.x) * blockDim.x + threadIdx.x) & ~i64{31}; k0 < n_chunks;
+       k0 += static_cast<i64>(gridDim.x) * blockDim.x) {
+    const i64 k = k0 + lane;
+    i64 n = 0;
+    if (k < n_chunks) n = chunk_off[k + 1] - chunk_off[k];
+    const bool mid = n > small_max && n <= mid_max;
+    const bool huge = n > small_max && !mid && n > kHugeChunk;
+    const bool big = n > small_max && !mid && !huge;
+    const u32 m_mid = __ballot_sync(0xffffffffu, mid);
+    const u32 m_huge = __ballot_sync(0xffffffffu, huge);
+    const u32 m_big = __ballot_sync(0xffffffffu, big);
+    int b_mid = 0, b_huge = 0, b_big = 0;
+    if (lane == 0) {
+      if (m_mid) b_mid = atomicAdd(&counters[0], __popc(m_mid));
+      if (m_huge) b_huge = atomicAdd(&counters[1], __popc(m_huge));
+      if (m_big) b_big = atomicAdd(&counters[2], __popc(m_big));
     }
-    seg_first[i] = lo;
+    b_mid = __shfl_sync(0xffffffffu, b_mid, 0);
+    b_huge = __shfl_sync(0xffffffffu, b_huge, 0);
+    b_big = __shfl_sync(0xffffffffu, b_big, 0);
+    if (mid) mid_list[b_mid + __popc(m_mid & lanemask_lt())] = static_cast<int32_t>(k);
+    if (huge) big_list[b_huge + __popc(m_huge & lanemask_lt())] = static_cast<int32_t>(k);
+    if (big) big_list[n_chunks - 1 - (b_big + __popc(m_big & lanemask_lt()))] = static_cast<int32_t>(k);
   }
 }
 
@@ -92,20 +75,6 @@ __global__ void k6_chunk_bases(const i64* __restrict__ chunk_nnz_off, i64 n_chun
        i += static_cast<i64>(gridDim.x) * blockDim.x) {
     const i64 r = i >> log2_chunks_per_row;
     chunk_base[i] = c_row_ptr[x_heavy[h0 + r]] + (chunk_nnz_off[i] - chunk_nnz_off[r << log2_chunks_per_row]);
-  }
-}
-
-// One product into the accumulator.  Measured on B200 (shared memory, 1024 threads per SM, products per clock
-// per SM): native integer atomics 12; floating-point atomicAdd 3.7 on uniform columns and 2.0 when a quarter of
-// the products hit 64 hot columns (a hand-written compare-and-swap loop was a third slower than the built-in); ranking equal columns first with a warp
-// match (match.any) only 0.5 — so there is no warp-level deduplication here, and the bitmap is tested before
-// it is set so that repeated columns cost a load instead of an atomic.
-template <typename V, bool NUMERIC>
-__device__ __forceinline__ void acc_add(bool valid, u32 cl, V v, V* acc, u32* bitmap) {
-  if (valid) {
-    if constexpr (NUMERIC) atomicAdd(&acc[cl], v);
-    const u32 bit = 1u << (cl & 31);
-    if (!(bitmap[cl >> 5] & bit)) atomicOr(&bitmap[cl >> 5], bit);
   }
 }
 
@@ -125,10 +94,6 @@ constexpr int kSmallMaxPerLane = GM_SMALL_PER_LANE;
 constexpr int kAccSmallChunk = 32 * kSmallMaxPerLane;
 constexpr int kSmallIdxBits = kSmallMaxPerLane == 32 ? 10 : (kSmallMaxPerLane == 16 ? 9 : 8);  // position of a product inside its chunk
 constexpr int kSmallWarps = 4;            // warps per block of the small-chunk kernel
-#ifndef GM_ACC_LIST_MIN
-#define GM_ACC_LIST_MIN 512
-#endif
-constexpr u32 kAccListMin = GM_ACC_LIST_MIN;  // chunks with more entries than this balance their dense words over the block
 
 // Sorts 32 * K packed keys, K per lane, element e = r * 32 + lane in key[r]; ascending in e afterwards.
 // Steps whose partner sits in another lane are the same instruction sequence for every step width, so they run
@@ -278,300 +243,464 @@ __global__ void __launch_bounds__(kSmallWarps * 32) k6_small_chunks(
   }
 }
 
-template <typename V, bool NUMERIC, int BT, int PT>
-__global__ void __launch_bounds__(BT, 1) k6_accumulate(
+
+// ---------------------------------------------------------------------------------------------------------
+// Mid-size chunks: one block of kMidThreads threads per chunk, symbolic pass then numeric pass.
+// Shared memory: bitmap (W/32 words) | rank of every word's first entry (16 bits each) | the chunk's values,
+// compact (mid_max entries).  A thread owns consecutive bitmap words and moves them with 16-byte accesses.
+// ---------------------------------------------------------------------------------------------------------
+constexpr int kMidPer = 8;                          // products a thread holds per tile
+constexpr int kMidTile = kMidThreads * kMidPer;     // 1024: chunks up to this size are read from HBM once
+
+inline size_t mid_smem_bytes(int W, int val_bytes, int mid_max) {
+  const size_t n_words = static_cast<size_t>(W) / 32;
+  return ((n_words * 6 + 15) & ~size_t{15}) + static_cast<size_t>(mid_max) * val_bytes + 64;
+}
+
+struct ChunkTask {
+  i64 k;       // chunk (batch-relative), -1: no more work
+  i64 lo, hi;  // its products in the staging buffer
+};
+
+// Work distribution: chunks are handed out by an atomic ticket over a list.  Getting from a ticket to the chunk's
+// products is a chain of three dependent global accesses (ticket, list entry, chunk bounds: two microseconds
+// end to end), and a block's barriers wait for the one thread that walks it.  So thread 0 keeps three tasks in
+// flight, one step of the chain each: at the start of a chunk it *issues* the ticket of the task three ahead, the
+// list read of the task two ahead and the bounds read of the next task, and it only touches the results when the
+// chunk's own work is done, by which time they have arrived.
+struct TaskPipe {
+  int* ticket;
+  int n_list, n_front;
+  const int32_t* list;
+  i64 list_flip;  // >= 0: list positions past n_front are read from the back (see k6_classify)
+  const i64* chunk_off;
+  int tk2 = 0;    // ticket of the task two ahead (arrived)
+  i64 k1 = -1;    // chunk of the next task (arrived)
+  int tk3 = 0;    // in flight during a chunk
+  i64 k2 = -1, lo1 = 0, hi1 = 0;
+
+  __device__ __forceinline__ i64 list_at(int t) const {
+    if (t >= n_list) return -1;
+    return (list_flip < 0 || t < n_front) ? list[t] : list[list_flip - (t - n_front)];
+  }
+  // fills `first` with the first task (blocking, once per block) and primes the pipe
+  __device__ __forceinline__ void start(ChunkTask* first) {
+    const int t0 = atomicAdd(ticket, 1);
+    const int t1 = atomicAdd(ticket, 1);
+    tk2 = atomicAdd(ticket, 1);
+    const i64 k0 = list_at(t0);
+    k1 = list_at(t1);
+    ChunkTask task{k0, 0, 0};
+    if (k0 >= 0) { task.lo = chunk_off[k0]; task.hi = chunk_off[k0 + 1]; }
+    *first = task;
+  }
+  __device__ __forceinline__ void issue() {  // start of a chunk
+    tk3 = atomicAdd(ticket, 1);
+    k2 = list_at(tk2);
+    if (k1 >= 0) { lo1 = chunk_off[k1]; hi1 = chunk_off[k1 + 1]; }
+  }
+  __device__ __forceinline__ void publish(ChunkTask* next) {  // when the chunk's products are done
+    *next = ChunkTask{k1, lo1, hi1};
+    k1 = k2;
+    tk2 = tk3;
+  }
+};
+
+template <typename V>
+__global__ void __launch_bounds__(kMidThreads) k6_mid_chunks(
     int32_t* x_col, V* x_val,            // staging buffer: products in, compacted chunks out (in place)
-    const i64* __restrict__ chunk_off,   // n_chunks + 1 batch-relative element offsets
-    i64 n_chunks, const i64* __restrict__ seg_first, i64 n_segs, int* __restrict__ ticket,
-    int log2_chunks_per_row, int W, int stages, int small_max,
-    u32* __restrict__ chunk_nnz,         // out, pre-zeroed: entries per chunk (empty chunks are never visited)
-    int* __restrict__ err) {
-  extern __shared__ __align__(128) unsigned char smem_acc_raw[];
-  constexpr int kAccTile = PT * BT;
-  constexpr int kAccMetaCap = BT;
+    const i64* __restrict__ chunk_off, const int32_t* __restrict__ mid_list, int* __restrict__ counters,
+    int log2_chunks_per_row, int W, int mid_max,
+    u32* __restrict__ chunk_nnz,         // out: entries per chunk
+    u64* __restrict__ totals) {          // [0] += products, [1] += entries of the chunks handled here (statistics)
+  extern __shared__ __align__(16) unsigned char smem_mid_raw[];
+  constexpr int T = kMidThreads;
   const int n_words = W >> 5;
-  // layout: [ring cols][ring vals][acc][dense-word list][bitmap][chunk offsets of the metadata window]
-  int32_t* r_col = reinterpret_cast<int32_t*>(smem_acc_raw);
-  V* r_val = reinterpret_cast<V*>(smem_acc_raw + static_cast<size_t>(stages) * kAccTile * 4);
-  unsigned char* after_ring = smem_acc_raw + static_cast<size_t>(stages) * kAccTile * (4 + (NUMERIC ? sizeof(V) : 0));
-  V* acc = reinterpret_cast<V*>(after_ring);
+  u32* bitmap = reinterpret_cast<u32*>(smem_mid_raw);                 // n_words
+  unsigned short* wpre = reinterpret_cast<unsigned short*>(bitmap + n_words);  // n_words: rank of the word's first entry
+  V* oval = reinterpret_cast<V*>(smem_mid_raw + ((static_cast<size_t>(n_words) * 6 + 15) & ~size_t{15}));
+  __shared__ u32 s_wsum[T / 32];
+  __shared__ ChunkTask s_task[2];
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const u32 wmask = static_cast<u32>(W - 1);
+  const u32 crow_mask = (1u << log2_chunks_per_row) - 1u;
+  const int log2W = 31 - __clz(W);
+  // every thread owns wpt consecutive bitmap words in the scan (eight for W = 32768: two 16-byte accesses)
+  const int wpt = n_words > T ? n_words / T : 1;
+  const int wb = tid * wpt;
+  const bool own = wb < n_words;
+
+  for (int w = tid; w < n_words; w += T) bitmap[w] = 0u;
+  for (int i = tid; i < mid_max; i += T) oval[i] = V(0);
+  TaskPipe pipe{&counters[3], counters[0], 0, mid_list, -1, chunk_off};
+  if (tid == 0) pipe.start(&s_task[0]);
+  __syncthreads();
+  u64 sum_n = 0, sum_m = 0;
+  int par = 0;
+  ChunkTask task = s_task[0];
+  // first tile of the first chunk
+  u32 c_reg[kMidPer];
+  auto load_cols = [&](const ChunkTask& tk, int tile) {
+#pragma unroll
+    for (int u = 0; u < kMidPer; ++u) {
+      const i64 q = tk.lo + static_cast<i64>(tile) * kMidTile + u * T + tid;
+      c_reg[u] = q < tk.hi ? static_cast<u32>(x_col[q]) & wmask : 0xffffffffu;
+    }
+  };
+  if (task.k >= 0) load_cols(task, 0);
+
+  while (task.k >= 0) {
+    const int n = static_cast<int>(task.hi - task.lo);
+    int32_t* const col = x_col + task.lo;
+    V* const val = x_val + task.lo;
+    const u32 col_base = (static_cast<u32>(task.k) & crow_mask) << log2W;
+    const int n_tiles = (n + kMidTile - 1) / kMidTile;
+    if (tid == 0) pipe.issue();
+
+    // ---- pass 1 (symbolic): mark the columns.  The values of the first tile are requested now, for pass 2.
+    V v_reg[kMidPer];
+#pragma unroll
+    for (int u = 0; u < kMidPer; ++u) {
+      const int q = u * T + tid;
+      if (q < n) v_reg[u] = val[q];
+    }
+    for (int tile = 0;;) {
+#pragma unroll
+      for (int u = 0; u < kMidPer; ++u)
+        if (c_reg[u] != 0xffffffffu) atomicOr(&bitmap[c_reg[u] >> 5], 1u << (c_reg[u] & 31));
+      if (++tile >= n_tiles) break;
+      load_cols(task, tile);
+    }
+    __syncthreads();
+    // ---- ranks: exclusive prefix over the words' populations
+    u32 pc = 0;
+    uint4 b0 = make_uint4(0, 0, 0, 0), b1 = b0;  // the usual case: eight words per thread
+    if (own) {
+      if (wpt == 8) {
+        b0 = *reinterpret_cast<const uint4*>(bitmap + wb);
+        b1 = *reinterpret_cast<const uint4*>(bitmap + wb + 4);
+        pc = __popc(b0.x) + __popc(b0.y) + __popc(b0.z) + __popc(b0.w) + __popc(b1.x) + __popc(b1.y) + __popc(b1.z) + __popc(b1.w);
+      } else {
+        for (int i = 0; i < wpt; ++i) pc += __popc(bitmap[wb + i]);
+      }
+    }
+    const u32 inc = warp_inclusive_scan(pc);
+    if (lane == 31) s_wsum[warp] = inc;
+    __syncthreads();
+    u32 ex = inc - pc, total = 0;
+#pragma unroll
+    for (int w = 0; w < T / 32; ++w) {
+      const u32 ws = s_wsum[w];
+      if (w < warp) ex += ws;
+      total += ws;
+    }
+    if (own) {
+      if (wpt == 8) {
+        u32 r0 = ex, r1 = r0 + __popc(b0.x), r2 = r1 + __popc(b0.y), r3 = r2 + __popc(b0.z), r4 = r3 + __popc(b0.w);
+        u32 r5 = r4 + __popc(b1.x), r6 = r5 + __popc(b1.y), r7 = r6 + __popc(b1.z);
+        *reinterpret_cast<uint4*>(wpre + wb) = make_uint4(r0 | (r1 << 16), r2 | (r3 << 16), r4 | (r5 << 16), r6 | (r7 << 16));
+      } else {
+        u32 run = ex;
+        for (int i = 0; i < wpt; ++i) {
+          wpre[wb + i] = static_cast<unsigned short>(run);
+          run += __popc(bitmap[wb + i]);
+        }
+      }
+    }
+    if (n_tiles > 1) load_cols(task, 0);  // (a single tile is still in registers)
+    __syncthreads();
+    // ---- pass 2 (numeric): every product to the slot of its column's rank
+    for (int tile = 0;;) {
+#pragma unroll
+      for (int u = 0; u < kMidPer; ++u) {
+        const u32 c = c_reg[u];
+        if (c != 0xffffffffu) {
+          const u32 r = static_cast<u32>(wpre[c >> 5]) + __popc(bitmap[c >> 5] & ((1u << (c & 31)) - 1u));
+          atomicAdd(&oval[r], v_reg[u]);
+        }
+      }
+      if (++tile >= n_tiles) break;
+      load_cols(task, tile);
+#pragma unroll
+      for (int u = 0; u < kMidPer; ++u) {
+        const int q = tile * kMidTile + u * T + tid;
+        if (q < n) v_reg[u] = val[q];
+      }
+    }
+    if (tid == 0) pipe.publish(&s_task[par ^ 1]);
+    __syncthreads();
+    // the next chunk's first columns are requested before this chunk is written out
+    const ChunkTask next = s_task[par ^ 1];
+    if (next.k >= 0) load_cols(next, 0);
+    // ---- write-out in place: columns from the bitmap (each thread its own words), values from the compact array
+    if (own && pc) {
+      u32 p = ex;
+      auto emit_word = [&](u32 bits, int w) {
+        const u32 cb = col_base + (static_cast<u32>(w) << 5);
+        while (bits) {
+          const int b = __ffs(bits) - 1;
+          bits &= bits - 1;
+          col[p++] = static_cast<int32_t>(cb + b);
+        }
+      };
+      if (wpt == 8) {
+        emit_word(b0.x, wb); emit_word(b0.y, wb + 1); emit_word(b0.z, wb + 2); emit_word(b0.w, wb + 3);
+        emit_word(b1.x, wb + 4); emit_word(b1.y, wb + 5); emit_word(b1.z, wb + 6); emit_word(b1.w, wb + 7);
+        *reinterpret_cast<uint4*>(bitmap + wb) = make_uint4(0, 0, 0, 0);
+        *reinterpret_cast<uint4*>(bitmap + wb + 4) = make_uint4(0, 0, 0, 0);
+      } else {
+        for (int i = 0; i < wpt; ++i) {
+          const u32 bits = bitmap[wb + i];
+          if (bits) {
+            bitmap[wb + i] = 0u;
+            emit_word(bits, wb + i);
+          }
+        }
+      }
+    }
+    for (int i = tid; i < static_cast<int>(total); i += T) {
+      val[i] = oval[i];
+      oval[i] = V(0);
+    }
+    if (tid == 0) {
+      chunk_nnz[task.k] = total;
+      sum_n += static_cast<u64>(n);
+      sum_m += total;
+    }
+    __syncthreads();
+    task = next;
+    par ^= 1;
+  }
+  if (tid == 0 && sum_n) {
+    atomicAdd(&totals[0], sum_n);
+    atomicAdd(&totals[1], sum_m);
+  }
+}
+
+// ---------------------------------------------------------------------------------------------------------
+// Big chunks: the dense accumulator.
+//
+// What binds this kernel is the shared-memory pipe (measured on B200 with a stream of products from HBM, products
+// per clock per SM: integer atomics >= 3, limited by the stream; floating-point add 2.1 on uniform columns, 1.7
+// with a bitmap test-and-set next to it), so a product costs one shared-memory operation, the floating-point atomic
+// add, and only the first product of a column pays a second one:
+//  * First-touch bitmap.  An idle slot holds -0.0, which is the identity of the addition, and a product that is a
+//    zero of either sign is added as +0.0; a slot that received anything is then never -0.0 again (x + (-x) rounds
+//    to +0.0).  The add returns the slot's old value, so the thread that sees -0.0 knows it was first and sets the
+//    column's bit with an integer atomic: one per entry of C instead of a load per product, structural zeros kept.
+//  * Bank spreading.  Columns of power-law matrices made by recursive quadrant picks have biased low bits
+//    (bit = 0 three times out of four), so a quarter of all products would land in bank 0: measured 1.1
+//    products per clock per SM, against 1.9 with the slot of a column rotated inside its group of 32 by a
+//    hash of the group index (bitmap words likewise).  The rotation is undone when the flush walks a group.
+// ---------------------------------------------------------------------------------------------------------
+#ifndef GM_ACC_LIST_MIN
+#define GM_ACC_LIST_MIN 512
+#endif
+constexpr u32 kAccListMin = GM_ACC_LIST_MIN;  // chunks with more entries than this balance their dense words over the block
+
+inline size_t acc_smem_bytes_big(int W, int val_bytes) {
+  const size_t n_words = static_cast<size_t>(W / 32);
+  return static_cast<size_t>(W) * val_bytes + n_words * 8 + ((n_words + 31) & ~size_t{31}) * 4 + 64;
+}
+
+template <typename V> struct Vec4;
+template <> struct Vec4<float> {
+  float4 d;
+  __device__ __forceinline__ void load(const float* p) { d = *reinterpret_cast<const float4*>(p); }
+  __device__ __forceinline__ float get(int u) const { return u == 0 ? d.x : u == 1 ? d.y : u == 2 ? d.z : d.w; }
+};
+template <> struct Vec4<double> {
+  double2 a, b;
+  __device__ __forceinline__ void load(const double* p) {
+    a = *reinterpret_cast<const double2*>(p);
+    b = *reinterpret_cast<const double2*>(p + 2);
+  }
+  __device__ __forceinline__ double get(int u) const { return u == 0 ? a.x : u == 1 ? a.y : u == 2 ? b.x : b.y; }
+};
+
+__device__ __forceinline__ float acc_idle(float) { return __uint_as_float(0x80000000u); }
+__device__ __forceinline__ double acc_idle(double) { return __longlong_as_double(static_cast<long long>(0x8000000000000000ull)); }
+__device__ __forceinline__ bool acc_touched(float x) { return __float_as_uint(x) != 0x80000000u; }
+__device__ __forceinline__ bool acc_touched(double x) { return static_cast<u64>(__double_as_longlong(x)) != 0x8000000000000000ull; }
+__device__ __forceinline__ float plus_zero(float v) { return __fadd_rn(v, 0.0f); }   // -0.0 -> +0.0, everything else unchanged
+__device__ __forceinline__ double plus_zero(double v) { return __dadd_rn(v, 0.0); }
+
+// rotation of a group of 32 columns inside the accumulator
+__device__ __forceinline__ u32 group_rot(u32 group) { return (group * 0x9E3779B1u) >> 27; }
+__device__ __forceinline__ u32 acc_slot(u32 cl) { return (cl & ~31u) | ((cl + group_rot(cl >> 5)) & 31u); }
+
+template <typename V, int BT>
+__global__ void __launch_bounds__(BT, 1024 / BT) k6_accumulate(
+    int32_t* x_col, V* x_val,            // staging buffer: products in, compacted chunks out (in place)
+    const i64* __restrict__ chunk_off, i64 n_chunks, const int32_t* __restrict__ big_list, int* __restrict__ counters,
+    int log2_chunks_per_row, int W,
+    u32* __restrict__ chunk_nnz) {       // out: entries per chunk
+  extern __shared__ __align__(128) unsigned char smem_acc_raw[];
+  const int n_words = W >> 5;
+  // layout: [acc][dense-word list][bitmap, whole groups of 32 words]
+  V* acc = reinterpret_cast<V*>(smem_acc_raw);
   // n_words entries {bits | word index, prefix}; W * sizeof(V) is a multiple of 128, so the list is 8-byte aligned
-  u64* dense_list = reinterpret_cast<u64*>(after_ring + (NUMERIC ? static_cast<size_t>(W) * sizeof(V) : 0));
+  u64* dense_list = reinterpret_cast<u64*>(smem_acc_raw + static_cast<size_t>(W) * sizeof(V));
   u32* bitmap = reinterpret_cast<u32*>(dense_list + n_words);
-  int* m_off = reinterpret_cast<int*>(bitmap + n_words);
-  __shared__ u64 full_bar[8];
   __shared__ u32 s_scan[33];
-  __shared__ i64 s_seg[2];
-  __shared__ int s_abort;
+  __shared__ ChunkTask s_task[2];
   __shared__ int s_dense_n[2];  // used by alternate chunks, so that resetting one needs no barrier of its own
 
+  constexpr int kWarps = BT / 32;
+  constexpr int kTile = 4 * BT;  // products per step: four consecutive ones per thread, two 16-byte loads
   const int tid = threadIdx.x, lane = tid & 31;
   const u32 wmask = static_cast<u32>(W - 1);
-  constexpr u32 kStageBytesCol = kAccTile * 4;
-  constexpr u32 kStageBytesVal = NUMERIC ? kAccTile * sizeof(V) : 0;
-  constexpr int kPerThread = kAccTile / BT;  // elements of a full tile per thread
-  constexpr int kWarps = BT / 32;
-  static_assert(kAccTile % BT == 0, "tile must be a multiple of the block");
-  // the flush gives every thread wpt consecutive bitmap words (wpt is a power of two, at most 32)
+  const u32 crow_mask = (1u << log2_chunks_per_row) - 1u;
+  const int log2W = 31 - __clz(W);
+  // the flush gives every thread wpt consecutive groups of 32 columns (wpt is a power of two, at most 32)
   const int wpt = n_words > BT ? n_words / BT : 1;
+  const V idle = acc_idle(V(0));
 
-  if (NUMERIC)
-    for (int s = tid; s < W; s += BT) acc[s] = V(0);
-  for (int w = tid; w < n_words; w += BT) bitmap[w] = 0u;
+  for (int s = tid; s < W; s += BT) acc[s] = idle;
+  for (int w = tid; w < ((n_words + 31) & ~31); w += BT) bitmap[w] = 0u;
+  TaskPipe pipe{&counters[4], counters[1] + counters[2], counters[1], big_list, n_chunks - 1, chunk_off};
   if (tid == 0) {
-    for (int s = 0; s < stages; ++s) mbar_init(&full_bar[s], 1);
-    s_abort = 0;
     s_dense_n[0] = 0;
     s_dense_n[1] = 0;
-    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    pipe.start(&s_task[0]);
   }
   __syncthreads();
-  u32 phase_bits = 0;  // bit s = parity to wait for on stage s
-  int dpar = 0;        // which dense-word counter the current chunk uses
-
-  for (;;) {
-    if (tid == 0) {
-      const int s = atomicAdd(ticket, 1);
-      s_seg[0] = s < n_segs ? seg_first[s] : -1;
-      s_seg[1] = s < n_segs ? seg_first[s + 1] : -1;
+  int dpar = 0;  // which dense-word counter the current chunk uses
+  int par = 0;
+  ChunkTask task = s_task[0];
+  // first tile of the first chunk: the stream starts at the 16-byte boundary below the chunk
+  int4 c4 = make_int4(0, 0, 0, 0);
+  Vec4<V> v4;
+  auto load_tile = [&](i64 p, i64 hi) {
+    if (p < hi) {
+      c4 = *reinterpret_cast<const int4*>(x_col + p);
+      v4.load(x_val + p);
     }
-    __syncthreads();
-    const i64 k_first = s_seg[0], k_end = s_seg[1];
-    __syncthreads();
-    if (k_first < 0) break;
-    if (k_first >= k_end) continue;
-    const i64 lo = chunk_off[k_first], hi = chunk_off[k_end];
-    if (lo >= hi) continue;
-    const i64 lo_al = lo & ~i64{3};  // 16-byte aligned start of the stream
-    const int n_tiles = static_cast<int>((hi - lo_al + kAccTile - 1) / kAccTile);
-    const int32_t* g_col = x_col + lo_al;
-    const V* g_val = x_val + lo_al;
+  };
+  if (task.k >= 0) load_tile((task.lo & ~i64{3}) + static_cast<i64>(tid) * 4, task.hi);
+  auto add = [&](u32 cl, V v) {
+    const V old = atomicAdd(&acc[acc_slot(cl)], plus_zero(v));
+    if (!acc_touched(old)) atomicOr(&bitmap[acc_slot(cl >> 5)], 1u << (cl & 31));  // first product of this column
+  };
 
-    auto issue = [&](int j, int st) {  // thread 0 only
-      const size_t g = static_cast<size_t>(j) * kAccTile;
-      mbar_expect_tx(&full_bar[st], kStageBytesCol + kStageBytesVal);
-      bulk_g2s(r_col + st * kAccTile, g_col + g, kStageBytesCol, &full_bar[st]);
-      if (NUMERIC) bulk_g2s(r_val + st * kAccTile, g_val + g, kStageBytesVal, &full_bar[st]);
-    };
-    if (tid == 0)
-      for (int j = 0; j < n_tiles && j < stages; ++j) issue(j, j);
+  while (task.k >= 0) {
+    const i64 lo = task.lo, hi = task.hi;
+    const u32 col_base = (static_cast<u32>(task.k) & crow_mask) << log2W;
+    if (tid == 0) pipe.issue();
 
-    // chunk metadata of the segment, refilled every kAccMetaCap chunks
-    i64 m0 = k_first;          // first chunk held in the metadata window
-    int kw = 0;                // current chunk = m0 + kw
-    const u32 crow_mask = (1u << log2_chunks_per_row) - 1u;
-    u32 crow = static_cast<u32>(k_first) & crow_mask;  // index of the current chunk inside its row (kept in step with kw)
-    const int log2W = 31 - __clz(W);
-    auto load_meta = [&]() {
-      for (int i = tid; i < kAccMetaCap; i += BT) {
-        const i64 kk = m0 + i;
-        if (kk <= k_end) m_off[i] = static_cast<int>(chunk_off[kk] - lo_al);
+    // ---- accumulate: the tile after the current one is already on its way while this one is added
+    for (i64 p = (lo & ~i64{3}) + static_cast<i64>(tid) * 4; p - static_cast<i64>(tid) * 4 < hi; p += kTile) {
+      const int4 c = c4;
+      const Vec4<V> v = v4;
+      load_tile(p + kTile, hi);
+      if (p >= lo && p + 3 < hi) {
+        add(static_cast<u32>(c.x) & wmask, v.get(0));
+        add(static_cast<u32>(c.y) & wmask, v.get(1));
+        add(static_cast<u32>(c.z) & wmask, v.get(2));
+        add(static_cast<u32>(c.w) & wmask, v.get(3));
+      } else if (p < hi) {
+        if (p >= lo) add(static_cast<u32>(c.x) & wmask, v.get(0));
+        if (p + 1 >= lo && p + 1 < hi) add(static_cast<u32>(c.y) & wmask, v.get(1));
+        if (p + 2 >= lo && p + 2 < hi) add(static_cast<u32>(c.z) & wmask, v.get(2));
+        if (p + 3 >= lo && p + 3 < hi) add(static_cast<u32>(c.w) & wmask, v.get(3));
       }
-    };
-    load_meta();
+    }
+    // ---- chunk complete: flush
     __syncthreads();
-
-    int pos = static_cast<int>(lo - lo_al);      // stream-relative position of the next element
-    const int end = static_cast<int>(hi - lo_al);
-    bool aborted = false;
-    int st = 0;
-
-    for (int j = 0; j < n_tiles; ++j) {
-      // ---- wait for the tile (bounded, with back-off so that the poll does not eat issue slots)
-      {
-        const u32 par = (phase_bits >> st) & 1u;
-        int spins = 0;
-        while (!mbar_try_wait(&full_bar[st], par)) {
-          __nanosleep(40);
-          if (*static_cast<volatile int*>(&s_abort)) break;  // somebody gave up: no tile will be issued any more
-          if (++spins > kAccSpinLimit) { s_abort = 1; break; }
-        }
-        phase_bits ^= (1u << st);
-      }
-      const int tile_lo = j * kAccTile;
-      const int tile_hi = min(end, tile_lo + kAccTile);
-      int32_t* tc = r_col + st * kAccTile - tile_lo;
-      V* tv = r_val + st * kAccTile - tile_lo;
-      while (pos < tile_hi) {
-        // make sure the current chunk and its end are inside the metadata window
-        if (kw + 33 >= kAccMetaCap) {  // the look-ahead below reads 32 chunks
-          __syncthreads();
-          m0 += kw;
-          kw = 0;
-          load_meta();
-          __syncthreads();
-        }
-        const int ce = m_off[kw + 1];
-        if (ce - m_off[kw] <= small_max) {
-          // an empty chunk, or a small one that the small-chunk kernel has dealt with: how many of the next 32
-          // chunks are like that?  Every warp evaluates the same shared-memory metadata, so the answer is
-          // uniform without a barrier.
-          const i64 kc = m0 + kw + lane;
-          const bool skip = kc < k_end && m_off[kw + lane + 1] - m_off[kw + lane] <= small_max;
-          const u32 not_skip = ~__ballot_sync(0xffffffffu, skip);
-          const int run = not_skip ? __ffs(not_skip) - 1 : 32;  // >= 1
-          kw += run;
-          crow = (crow + static_cast<u32>(run)) & crow_mask;
-          pos = m_off[kw];
-          continue;
-        }
-        const int sub_hi = min(tile_hi, ce);
-        const u32 col_base = crow << log2W;
-        if (!s_abort) {
-          for (int base = pos; base < sub_hi; base += BT * kPerThread) {
-            // slots of this warp that still hold products of the sub-range (warp-uniform): a short sub-range
-            // must not pay for the whole unrolled body
-            const int wq = base + (tid & ~31);
-            const int nu = wq >= sub_hi ? 0 : min(kPerThread, (sub_hi - wq + BT - 1) / BT);
-            if (nu == kPerThread && wq + (kPerThread - 1) * BT + 32 <= sub_hi) {
-              u32 cl[kPerThread];
-              V v[kPerThread];
-#pragma unroll
-              for (int u = 0; u < kPerThread; ++u) {
-                const int q = base + u * BT + tid;
-                cl[u] = static_cast<u32>(tc[q]) & wmask;
-                if (NUMERIC) v[u] = tv[q];
-              }
-#pragma unroll
-              for (int u = 0; u < kPerThread; ++u) acc_add<V, NUMERIC>(true, cl[u], v[u], acc, bitmap);
-            } else {
-              for (int u = 0; u < nu; ++u) {
-                const int q = base + u * BT + tid;
-                if (q < sub_hi) acc_add<V, NUMERIC>(true, static_cast<u32>(tc[q]) & wmask, NUMERIC ? tv[q] : V(0), acc, bitmap);
-              }
-            }
-          }
-        }
-        pos = sub_hi;
-        if (pos < ce) break;  // chunk continues in the next tile
-        // ---- chunk complete: flush
-        __syncthreads();
-        const int wb = tid * wpt;
-        const bool warp_has_words = (tid & ~31) * wpt < n_words;  // warp-uniform
-        u32 pc = 0;
-        u32 word0 = 0;  // the thread's first (for wpt == 1: only) word stays in a register
-        if (wb < n_words) {
-          word0 = bitmap[wb];
-          pc = __popc(word0);
-          for (int i = 1; i < wpt; ++i) pc += __popc(bitmap[wb + i]);
-        }
-        // Block-wide exclusive prefix with one barrier: every warp publishes its sum, then adds up the sums of
-        // the warps before it (and all of them, for the chunk's entry count) on its own.
-        const u32 inc = warp_inclusive_scan(pc);
-        if (lane == 31) s_scan[tid >> 5] = inc;
-        __syncthreads();
-        const u32 wsum = lane < kWarps ? s_scan[lane] : 0u;
-        const u32 total = __reduce_add_sync(0xffffffffu, wsum);
-        u32 ex = __reduce_add_sync(0xffffffffu, lane < (tid >> 5) ? wsum : 0u) + inc - pc;
-        if (tid == 0) chunk_nnz[m0 + kw] = total;
-        {
-          // in place: the chunk's products [m_off[kw], ce) are all in shared memory or consumed by now
-          int32_t* const c_col = x_col + lo_al + m_off[kw];
-          V* const c_val = x_val + lo_al + m_off[kw];
-          // Words with few bits are written by their owner.  In a chunk with many entries the dense words
-          // cluster at the low end (hub columns), i.e. in the first warps, so they go to a list that all warps
-          // then share out evenly; there the 32 lanes of a warp write one word at a time.  A chunk with few
-          // entries cannot be far out of balance and skips the list and its barrier.
-          const bool use_list = total > kAccListMin;  // block-uniform
-          if (warp_has_words) {
-            for (int i = 0; i < wpt; ++i) {
-              const u32 word = i == 0 ? word0 : (wb + i < n_words ? bitmap[wb + i] : 0u);
-              const u32 wpc = __popc(word);
-              const bool dense = use_list && wpc > 4;
-              if (use_list) {
-                const u32 dmask = __ballot_sync(0xffffffffu, dense);
-                if (dmask) {
-                  int lbase = 0;
-                  if (lane == 0) lbase = atomicAdd(&s_dense_n[dpar], __popc(dmask));
-                  lbase = __shfl_sync(0xffffffffu, lbase, 0);
-                  if (dense)  // {bits, word index, prefix} in one entry: the write-out needs a single load
-                    dense_list[lbase + __popc(dmask & lanemask_lt())] =
-                        (static_cast<u64>((static_cast<u32>(wb + i) << 16) | ex) << 32) | word;
-                }
-              }
-              if (!dense && wpc) {
-                u32 wbits = word;
-                u32 p = ex;
-                while (wbits) {
-                  const int b = __ffs(wbits) - 1;
-                  wbits &= wbits - 1;
-                  const int slot = ((wb + i) << 5) + b;
-                  c_col[p] = static_cast<int32_t>(col_base + slot);
-                  c_val[p] = acc[slot];
-                  acc[slot] = V(0);
-                  ++p;
-                }
-              }
-              if (wpc) bitmap[wb + i] = 0u;  // a listed word's bits travel in its list entry
-              ex += wpc;
-            }
-          }
+    if (tid == 0) pipe.publish(&s_task[par ^ 1]);  // read after the next barrier
+    const int wb = tid * wpt;
+    const bool warp_has_words = (tid & ~31) * wpt < n_words;  // warp-uniform
+    u32 pc = 0;
+    u32 word0 = 0;  // the thread's first (for wpt == 1: only) word stays in a register
+    if (wb < n_words) {
+      word0 = bitmap[acc_slot(static_cast<u32>(wb))];
+      pc = __popc(word0);
+      for (int i = 1; i < wpt; ++i) pc += __popc(bitmap[acc_slot(static_cast<u32>(wb + i))]);
+    }
+    // Block-wide exclusive prefix with one barrier: every warp publishes its sum, then adds up the sums of
+    // the warps before it (and all of them, for the chunk's entry count) on its own.
+    const u32 inc = warp_inclusive_scan(pc);
+    if (lane == 31) s_scan[tid >> 5] = inc;
+    __syncthreads();
+    const u32 wsum = lane < kWarps ? s_scan[lane] : 0u;
+    const u32 total = __reduce_add_sync(0xffffffffu, wsum);
+    u32 ex = __reduce_add_sync(0xffffffffu, lane < (tid >> 5) ? wsum : 0u) + inc - pc;
+    if (tid == 0) chunk_nnz[task.k] = total;
+    // the next chunk's first tile is requested before this chunk is written out
+    const ChunkTask next = s_task[par ^ 1];
+    if (next.k >= 0) load_tile((next.lo & ~i64{3}) + static_cast<i64>(tid) * 4, next.hi);
+    {
+      // in place: the chunk's products have all been consumed by now
+      int32_t* const c_col = x_col + lo;
+      V* const c_val = x_val + lo;
+      // Groups with few entries are written by their owner.  In a chunk with many entries the dense groups
+      // cluster at the low end (hub columns), i.e. in the first warps, so they go to a list that all warps
+      // then share out evenly; there the 32 lanes of a warp write one group at a time.  A chunk with few
+      // entries cannot be far out of balance and skips the list and its barrier.
+      const bool use_list = total > kAccListMin;  // block-uniform
+      if (warp_has_words) {
+        for (int i = 0; i < wpt; ++i) {
+          const u32 word = i == 0 ? word0 : (wb + i < n_words ? bitmap[acc_slot(static_cast<u32>(wb + i))] : 0u);
+          const u32 wpc = __popc(word);
+          const bool dense = use_list && wpc > 4;
           if (use_list) {
-            __syncthreads();
-            const int n_dense = s_dense_n[dpar];
-            auto emit = [&](u64 e) {
-              const u32 word = static_cast<u32>(e);
-              if ((word >> lane) & 1u) {
-                const u32 hi32 = static_cast<u32>(e >> 32);
-                const int slot = static_cast<int>((hi32 >> 16) << 5) + lane;
-                const u32 p = (hi32 & 0xffffu) + __popc(word & lanemask_lt());
-                c_col[p] = static_cast<int32_t>(col_base + slot);
-                c_val[p] = acc[slot];
-                acc[slot] = V(0);
-              }
-            };
-            for (int i = tid >> 5; i < n_dense; i += 2 * kWarps) {  // two words in flight per warp
-              const u64 e0 = dense_list[i];
-              const bool two = i + kWarps < n_dense;
-              const u64 e1 = two ? dense_list[i + kWarps] : 0ull;
-              emit(e0);
-              emit(e1);
+            const u32 dmask = __ballot_sync(0xffffffffu, dense);
+            if (dmask) {
+              int lbase = 0;
+              if (lane == 0) lbase = atomicAdd(&s_dense_n[dpar], __popc(dmask));
+              lbase = __shfl_sync(0xffffffffu, lbase, 0);
+              if (dense)  // {bits, group index, prefix} in one entry: the write-out needs a single load
+                dense_list[lbase + __popc(dmask & lanemask_lt())] =
+                    (static_cast<u64>((static_cast<u32>(wb + i) << 16) | ex) << 32) | word;
             }
-            if (tid == 0) s_dense_n[dpar ^ 1] = 0;  // next list's counter: last read two barriers ago
-            dpar ^= 1;
           }
+          if (!dense && wpc) {
+            u32 wbits = word;
+            u32 p = ex;
+            const u32 rot = group_rot(static_cast<u32>(wb + i));
+            while (wbits) {
+              const int b = __ffs(wbits) - 1;
+              wbits &= wbits - 1;
+              const int slot = ((wb + i) << 5) + static_cast<int>((static_cast<u32>(b) + rot) & 31u);
+              c_col[p] = static_cast<int32_t>(col_base + ((wb + i) << 5) + b);
+              c_val[p] = acc[slot];
+              acc[slot] = idle;
+              ++p;
+            }
+          }
+          if (wpc) bitmap[acc_slot(static_cast<u32>(wb + i))] = 0u;  // a listed word's bits travel in its list entry
+          ex += wpc;
         }
+      }
+      if (use_list) {
         __syncthreads();
-        ++kw;
-        crow = (crow + 1u) & crow_mask;
-      }
-      // ---- the stage is free again once every warp has finished the tile.  Only the warp that refills it has to
-      // wait for that: the others announce that they are done (named barrier 1 + stage) and go on to the next
-      // tile, whose data is in another stage.  A warp cannot arrive twice on a barrier before it has completed:
-      // its next use of this stage waits for the refill, which is issued after the barrier.
-      // (Only for the block that has an SM to itself: the named barriers of narrower blocks, several per SM, would
-      // not fit the SM's sixteen.)
-      if constexpr (BT == 1024) {
-        if (j + stages < n_tiles) {  // (uniform)
-          if (tid < 32) {
-            asm volatile("bar.sync %0, %1;" ::"r"(1 + st), "r"(BT) : "memory");
-            if (tid == 0 && !*static_cast<volatile int*>(&s_abort)) issue(j + stages, st);
-          } else {
-            asm volatile("bar.arrive %0, %1;" ::"r"(1 + st), "r"(BT) : "memory");
+        const int n_dense = s_dense_n[dpar];
+        auto emit = [&](u64 e) {
+          const u32 word = static_cast<u32>(e);
+          if ((word >> lane) & 1u) {
+            const u32 hi32 = static_cast<u32>(e >> 32);
+            const u32 grp = hi32 >> 16;
+            const int slot = static_cast<int>((grp << 5) + ((static_cast<u32>(lane) + group_rot(grp)) & 31u));
+            const u32 p = (hi32 & 0xffffu) + __popc(word & lanemask_lt());
+            c_col[p] = static_cast<int32_t>(col_base + (grp << 5) + lane);
+            c_val[p] = acc[slot];
+            acc[slot] = idle;
           }
+        };
+        for (int i = tid >> 5; i < n_dense; i += 2 * kWarps) {  // two groups in flight per warp
+          const u64 e0 = dense_list[i];
+          const bool two = i + kWarps < n_dense;
+          const u64 e1 = two ? dense_list[i + kWarps] : 0ull;
+          emit(e0);
+          emit(e1);
         }
-      } else {
-        __syncthreads();
-        if (tid == 0 && j + stages < n_tiles && !*static_cast<volatile int*>(&s_abort)) issue(j + stages, st);
+        if (tid == 0) s_dense_n[dpar ^ 1] = 0;  // next list's counter: last read two barriers ago
+        dpar ^= 1;
       }
-      st = (st + 1 == stages) ? 0 : st + 1;
     }
-    __syncthreads();  // every warp is through the segment
-    aborted = s_abort != 0;
-    if (aborted) {
-      // Tiles that were issued but not consumed still target this block's shared memory: give each a
-      // bounded chance to land before the block exits (its barrier answers at once if it already did).
-      if (tid == 0) {
-        dev_set_error(err, kDevTimeout);
-        for (int s2 = 0; s2 < stages; ++s2) {
-          int spins = 0;
-          while (!mbar_try_wait(&full_bar[s2], (phase_bits >> s2) & 1u) && ++spins < (1 << 20)) {
-          }
-        }
-      }
-      __syncthreads();
-      return;
-    }
+    __syncthreads();
+    task = next;
+    par ^= 1;
   }
 }
 

@@ -15,21 +15,13 @@ size_t light_smem_bytes(int64_t slots, int64_t cap, int val_bytes, bool numeric)
   return b;
 }
 
-int acc_block_threads(int ctas_per_sm, size_t smem_budget, int val_bytes) {
-  int bt = 1024 / ctas_per_sm;  // two products per thread and tile: see the accumulate kernel
-  // metadata window + three ring stages may take at most half of the budget; the rest is the accumulator
-  while (bt > 128 && static_cast<size_t>(bt) * 12 + 3 * 2 * static_cast<size_t>(bt) * (4 + val_bytes) > smem_budget / 2) bt /= 2;
-  return bt;
-}
+int acc_block_threads(int ctas_per_sm) { return 1024 / ctas_per_sm; }
 
-size_t acc_smem_bytes(int64_t W, int val_bytes, bool numeric, int block_threads) {
-  // bitmap (1 bit per column, twice) + (numeric: one value per column), plus what the streaming needs at
-  // least: the chunk-metadata window (one entry per thread) and three ring stages of two products per thread
-  const size_t bt = static_cast<size_t>(block_threads);
+size_t acc_smem_bytes(int64_t W, int val_bytes, bool numeric) {
+  // bitmap (1 bit per column) + an 8-byte list entry per bitmap word (flush) + (numeric: one value per column);
+  // a fifth of the column bytes is kept back for the kernels' other tables
   size_t b = static_cast<size_t>(W / 32) * 12 + 256;
-  b += bt * (numeric ? 12 : 4);
-  b += 3 * 2 * bt * (numeric ? 4 + val_bytes : 4);
-  if (numeric) b += static_cast<size_t>(W) * val_bytes;
+  if (numeric) b += static_cast<size_t>(W) * val_bytes + static_cast<size_t>(W) * val_bytes / 5;
   return b;
 }
 
@@ -61,11 +53,10 @@ int planner_params(int64_t c_cols, int dtype, size_t smem_bytes, const gm_plan_o
   if (ctas != 1 && ctas != 2 && ctas != 4 && ctas != 8) return GM_ERR_INVALID_ARG;
   out->acc_ctas_per_sm = ctas;
   const int64_t acc_budget = S / ctas - reserve;
-  const int bt = acc_block_threads(ctas, static_cast<size_t>(acc_budget), sv);
-  out->acc_block_threads = bt;
+  out->acc_block_threads = acc_block_threads(ctas);
   int64_t W = 32;
-  while (static_cast<int64_t>(acc_smem_bytes(W * 2, sv, true, bt)) <= acc_budget && W < (int64_t{1} << 30)) W *= 2;
-  if (static_cast<int64_t>(acc_smem_bytes(W, sv, true, bt)) > acc_budget) return GM_ERR_UNSUPPORTED_SMEM;
+  while (static_cast<int64_t>(acc_smem_bytes(W * 2, sv, true)) <= acc_budget && W < (int64_t{1} << 30)) W *= 2;
+  if (static_cast<int64_t>(acc_smem_bytes(W, sv, true)) > acc_budget) return GM_ERR_UNSUPPORTED_SMEM;
   if (o.chunk_width) {
     const int64_t w = o.chunk_width;
     if (w < 32 || (w & (w - 1)) || w > W) return GM_ERR_INVALID_ARG;

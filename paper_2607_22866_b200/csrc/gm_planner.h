@@ -9,9 +9,8 @@ namespace gm {
 
 constexpr int kMultisplitBinCap = 2048;  // (parent, child) bins one multisplit tile keeps in smem
 constexpr int kMinSmemBytes = 16384;
-// threads of one accumulate block when `ctas_per_sm` of them share an SM (1024 threads per SM in total)
-// (fewer when the shared-memory budget is too small for the ring and metadata of a wide block)
-int acc_block_threads(int ctas_per_sm, size_t smem_budget, int val_bytes);
+// threads of one dense-accumulator block when `ctas_per_sm` of them share an SM (1024 threads per SM in total)
+int acc_block_threads(int ctas_per_sm);
 
 inline int ilog2_floor(uint64_t x) {
   int l = 0;
@@ -34,7 +33,7 @@ int planner_params(int64_t c_cols, int dtype, size_t smem_bytes, const gm_plan_o
 // `cap` (power of two) output entries.
 size_t light_smem_bytes(int64_t slots, int64_t cap, int val_bytes, bool numeric);
 // Shared memory one chunk accumulator of width W needs.
-size_t acc_smem_bytes(int64_t W, int val_bytes, bool numeric, int block_threads);
+size_t acc_smem_bytes(int64_t W, int val_bytes, bool numeric);
 
 struct Batch {
   int64_t h0, h1;      // heavy rows [h0, h1) (positions in the heavy-row list)
