@@ -497,6 +497,10 @@ __global__ void __launch_bounds__(kMidThreads) k6_mid_chunks(
 #define GM_ACC_LIST_MIN 512
 #endif
 constexpr u32 kAccListMin = GM_ACC_LIST_MIN;  // chunks with more entries than this balance their dense words over the block
+#ifndef GM_ACC_DENSE_MIN
+#define GM_ACC_DENSE_MIN 4
+#endif
+constexpr u32 kAccDenseMin = GM_ACC_DENSE_MIN;  // a group with more entries than this is written by a whole warp
 
 inline size_t acc_smem_bytes_big(int W, int val_bytes) {
   const size_t n_words = static_cast<size_t>(W / 32);
@@ -642,7 +646,7 @@ __global__ void __launch_bounds__(BT, 1024 / BT) k6_accumulate(
         for (int i = 0; i < wpt; ++i) {
           const u32 word = i == 0 ? word0 : (wb + i < n_words ? bitmap[acc_slot(static_cast<u32>(wb + i))] : 0u);
           const u32 wpc = __popc(word);
-          const bool dense = use_list && wpc > 4;
+          const bool dense = use_list && wpc > kAccDenseMin;
           if (use_list) {
             const u32 dmask = __ballot_sync(0xffffffffu, dense);
             if (dmask) {
