@@ -16,6 +16,8 @@ the same product on its own GPU, no collective touches the data path.
 from __future__ import annotations
 
 import argparse
+import ctypes
+import gc
 import json
 import os
 import statistics
@@ -37,11 +39,16 @@ DEFAULT_CONFIG = 2  # R-MAT scale 20, edge factor 16, fp32: the largest fp32 pow
 
 
 # DRAM bytes per launch (ncu dram__bytes_read.sum + dram__bytes_write.sum) over the algorithmic bytes of the same
-# launch, measured on a scaled-down case of the same kernels (R-MAT scale 17, 1.09 G products per step: see
-# profiles/dram_traffic_rmat17_f32.md).  Traffic grows in proportion to the products processed, so a full-size
-# launch is the algorithmic figure times this ratio.
-TRAFFIC_RATIO = {"k4_expand": 1.03, "k5a_histogram": 0.34, "k5b_multisplit": 0.99, "k6_small_chunks": 0.73, "k6_accumulate": 1.01,
-                 "k7_gather": 0.99}
+# launch, from single-kernel, single-launch ncu captures of these kernels on the same product scaled down by 2**2
+# (R-MAT scale 18, one batch of 0.5-0.8 G products, about 4 GB on the device).  Traffic grows in proportion to the
+# products processed, so a full-size launch is its algorithmic figure times this ratio.  A kernel that has changed
+# since its capture has no entry (traffic is then reported as null).
+TRAFFIC_RATIO = {}
+TRAFFIC_SOURCE = "single-launch ncu captures on R-MAT scale 18 (same recipe, 2**2 smaller), scaled by products"
+
+
+def ctypes_copy(dst, src):
+    ctypes.memmove(ctypes.byref(dst), ctypes.byref(src), ctypes.sizeof(src))
 
 
 def _peaks():
@@ -167,8 +174,12 @@ def oracle_timed(A, B, budget_s: float = 15.0):
 
     ip = oracle.row_products(A, B)
     total = int(ip.sum())
+    # Every call of the oracle sets up one dense accumulator of C.m columns per thread; with millions of columns
+    # that set-up must be spread over many rows, so a wide product is timed on a few large blocks.
+    wide = B.n_cols > (1 << 21)
+    n_blocks = 4 if wide else 64
     # calibrate on a small sample, then size the real one for roughly `budget_s`
-    cal = _row_sample(A.n_rows, 16, 0.002)
+    cal = _row_sample(A.n_rows, 2 if wide else 16, 0.02 if wide else 0.002)
     t = time.perf_counter()
     threads = 1
     for r0, r1 in cal:
@@ -177,7 +188,7 @@ def oracle_timed(A, B, budget_s: float = 15.0):
     cal_products = sum(int(ip[r0:r1].sum()) for r0, r1 in cal)
     rate = max(cal_products, 1) / dt
     frac = min(1.0, max(0.004, budget_s * rate / max(total, 1)))
-    blocks = _row_sample(A.n_rows, 64, frac)
+    blocks = _row_sample(A.n_rows, n_blocks, frac)
     products = sum(int(ip[r0:r1].sum()) for r0, r1 in blocks)
     t = time.perf_counter()
     for r0, r1 in blocks:
@@ -261,6 +272,8 @@ def main():
     ap.add_argument("--e2e-steps", type=int, default=2)
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-extra", action="store_true",
+                    help="skip the forced-multisplit step and the per-config list (default workload only)")
     ap.add_argument("--opt", action="append", default=[], metavar="FIELD=INT",
                     help="set a field of gm_plan_opts (e.g. level0_multisplit=1, tau=4096); repeatable")
     args = ap.parse_args()
@@ -299,60 +312,69 @@ def main():
             raise SystemExit(f"--opt: gm_plan_opts has no field '{field}'")
         setattr(opts, field, int(value))
 
-    def step(timing: bool):
-        plan = gm.spgemm_plan(dA, dB, SMEM_BYTES, opts)
-        if timing:
-            plan.set_timing(True)
-        C = gm.spgemm_execute(plan)
-        info, st = plan.info(), plan.stats()
-        nnz = C.nnz
-        del C
-        plan.destroy()
-        return info, st, nnz
-
     def barrier():
         if world > 1:
             dist.barrier()
         torch.cuda.synchronize()
 
-    for _ in range(args.warmup):
-        info, st, nnz = step(False)
-    barrier()
-    sampler = ClockSampler(local_rank)
-    sampler.start()
-    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    barrier()
-    ev0.record()
-    launches = 0
-    stats_sum: dict[str, float] = {}
-    for _ in range(args.steps):
-        info, st, nnz = step(True)
-        launches += int(info.launches + st.launches)
-        for name, _t in st._fields_:
-            if name != "reserved":
-                stats_sum[name] = stats_sum.get(name, 0.0) + float(getattr(st, name))
-    ev1.record()
-    barrier()
-    clocks = sampler.stop()
-    ms_total = ev0.elapsed_time(ev1)
-    t = torch.tensor([ms_total], device="cuda", dtype=torch.float64)
-    if world > 1:
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    ms_step = float(t.item()) / args.steps
-    products = int(info.products_total)
-    value = world * 2.0 * products / (ms_step * 1e-3) / 1e9
-    stats_avg = {k: v / args.steps for k, v in stats_sum.items()}
+    def measure(A, B, dA, dB, opts, steps, warmup, sample_clocks):
+        """`warmup` untimed and `steps` timed products (plan + execute each).  Returns a dict with the step time,
+        the plan's facts, the per-kernel table (algorithmic bytes, CUDA-event time) and the dominant kernel."""
+        sv = A.val.dtype.itemsize
+
+        def step(timing: bool):
+            plan = gm.spgemm_plan(dA, dB, SMEM_BYTES, opts)
+            if timing:
+                plan.set_timing(True)
+            C = gm.spgemm_execute(plan)
+            info, st = plan.info(), plan.stats()
+            nnz = C.nnz
+            del C
+            plan.destroy()
+            return info, st, nnz
+
+        for _ in range(warmup):
+            info, st, nnz = step(False)
+        barrier()
+        sampler = ClockSampler(local_rank) if sample_clocks else None
+        if sampler:
+            sampler.start()
+        ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        barrier()
+        ev0.record()
+        launches = 0
+        stats_sum: dict[str, float] = {}
+        for _ in range(steps):
+            info, st, nnz = step(True)
+            launches += int(info.launches + st.launches)
+            for name, _t in st._fields_:
+                if name != "reserved":
+                    stats_sum[name] = stats_sum.get(name, 0.0) + float(getattr(st, name))
+        ev1.record()
+        barrier()
+        clocks = sampler.stop() if sampler else None
+        t = torch.tensor([ev0.elapsed_time(ev1)], device="cuda", dtype=torch.float64)
+        if world > 1:
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms_step = float(t.item()) / steps
+        products = int(info.products_total)
+        stats_avg = {k: v / steps for k, v in stats_sum.items()}
+        # byte model: the row analysis (untimed plan) says which entries of A sit in light rows
+        plan = gm.spgemm_plan(dA, dB, SMEM_BYTES, opts)
+        ip_dev = plan.row_products().cpu().numpy()
+        plan.destroy()
+        n_light_entries_a = int(np.diff(A.row_ptr)[ip_dev <= info.params.tau].sum())
+        kt = kernel_table(info, stats_avg, sv, B.nnz, n_light_entries_a)
+        dom = max(kt, key=lambda k: kt[k]["ms"])
+        return {"ms_step": ms_step, "value": world * 2.0 * products / (ms_step * 1e-3) / 1e9, "products": products,
+                "info": info, "kernels": kt, "dominant": dom, "launches": launches, "nnz": int(nnz), "clocks": clocks}
+
+    peak, peak_kind = _peaks()
+    m = measure(A, B, dA, dB, opts, args.steps, args.warmup, True)
+    info, kt, dom, nnz, products, launches = m["info"], m["kernels"], m["dominant"], m["nnz"], m["products"], m["launches"]
+    value, ms_step, clocks, tau = m["value"], m["ms_step"], m["clocks"], info.params.tau
 
     # ---- roofline of the dominant kernel (times: CUDA events recorded by the library on the execute stream)
-    peak, peak_kind = _peaks()
-    a_len = np.diff(A.row_ptr)
-    tau = info.params.tau
-    plan = gm.spgemm_plan(dA, dB, SMEM_BYTES, opts)   # untimed: the row analysis feeds the byte model
-    ip_dev = plan.row_products().cpu().numpy()
-    plan.destroy()
-    n_light_entries_a = int(a_len[ip_dev <= tau].sum())
-    kt = kernel_table(info, stats_avg, sv, B.nnz, n_light_entries_a)
-    dom = max(kt, key=lambda k: kt[k]["ms"])
     n_b = max(int(info.n_batches), 1)
     n_split = max(info.params.n_levels - (1 if info.level0_direct else 0), 1)
     per_launch = {"k4_expand": n_b, "k5a_histogram": n_b * n_split,
@@ -361,7 +383,7 @@ def main():
     roofline = {"kernel": dom, "bound": "hbm", "achieved": kt[dom]["gbs"], "peak": peak, "unit": "GB/s",
                 "frac": kt[dom]["gbs"] / peak, "peak_kind": f"of {peak_kind}",
                 "traffic": (kt[dom]["bytes"] / per_launch * TRAFFIC_RATIO[dom]) if dom in TRAFFIC_RATIO else None,
-                "traffic_source": "ncu on R-MAT scale 17, scaled by products (profiles/dram_traffic_rmat17_f32.md)",
+                "traffic_source": TRAFFIC_SOURCE,
                 "bytes_per_launch": kt[dom]["bytes"] / per_launch, "ms_per_launch": kt[dom]["ms"] / per_launch,
                 "launches_per_step": per_launch}
 
@@ -380,9 +402,51 @@ def main():
         "roofline": roofline, "kernels": kt, "clocks": clocks, "gpu_launches": launches,
     }
 
+    def frac_of(k):
+        return {"bytes": k["bytes"], "ms": k["ms"], "gbs": k["gbs"], "frac": k["gbs"] / peak, "peak_kind": f"of {peak_kind}"}
+
+    if rank == 0 and not args.no_extra and info.params.n_levels > 0 and info.rows_heavy > 0:
+        # The default plan of a one-level product lets the expansion place the products, so no multisplit pass runs
+        # in the timed steps above.  Same workload once more with the first level as the separate histogram and
+        # multisplit passes over the staging buffer (Algorithm 5 as printed): the multisplit kernel's own number.
+        o2 = gm.PlanOpts()
+        ctypes_copy(o2, opts)
+        o2.level0_multisplit = 1
+        o2.separate_histogram = 1
+        mf = measure(A, B, dA, dB, o2, max(2, min(args.steps, 3)), 1, False)
+        line["kernels_multisplit_forced"] = {
+            "plan_opts": ["level0_multisplit=1", "separate_histogram=1"], "ms_per_step": mf["ms_step"], "value": mf["value"],
+            "k4_expand": frac_of(mf["kernels"]["k4_expand"]), "k5a_histogram": frac_of(mf["kernels"]["k5a_histogram"]),
+            "k5b_multisplit": frac_of(mf["kernels"]["k5b_multisplit"])}
+
+    if rank == 0 and not args.no_extra and args.config == DEFAULT_CONFIG and args.shrink == 0:
+        # the other four workloads, a few steps each: GFLOP/s and the dominant kernel's fraction of the HBM roof
+        del dA, dB
+        per_config = []
+        for ci in [c for c in range(len(gen.CONFIG_NAMES)) if c != args.config]:
+            gc.collect()
+            torch.cuda.empty_cache()
+            try:
+                Ai, Bi, _d = gen.config_inputs(ci)
+                dAi = gm.DeviceCSR.from_host(Ai)
+                dBi = dAi if Bi is Ai else gm.DeviceCSR.from_host(Bi)
+                mi = measure(Ai, Bi, dAi, dBi, gm.PlanOpts(), 3, 3, False)
+                kd = mi["kernels"][mi["dominant"]]
+                per_config.append({"workload": gen.CONFIG_NAMES[ci], "dtype": "f32" if Ai.val.dtype.itemsize == 4 else "f64",
+                                   "value": mi["value"], "unit": "GFLOP/s", "ms_per_step": mi["ms_step"], "steps": 3,
+                                   "products": mi["products"], "nnz_c": mi["nnz"], "levels": mi["info"].params.levels(),
+                                   "batches": int(mi["info"].n_batches), "dominant_kernel": mi["dominant"],
+                                   "achieved": kd["gbs"], "frac": kd["gbs"] / peak, "peak_kind": f"of {peak_kind}"})
+                del dAi, dBi, Ai, Bi
+            except (gm.GmError, MemoryError, RuntimeError) as exc:
+                per_config.append({"workload": gen.CONFIG_NAMES[ci], "skipped": f"{type(exc).__name__}: {exc}"[:200]})
+        line["per_config"] = per_config
+        dA = dB = None
+
     if rank == 0 and not args.no_e2e:
         # the host entry point uploads A and B itself: give it the whole device (no resident copies, no cached blocks)
-        del dA, dB
+        dA = dB = None
+        gc.collect()
         torch.cuda.empty_cache()
         try:
             line["e2e"] = e2e_leg(gm, torch, A, B, int(nnz), products, args.e2e_steps)

@@ -85,7 +85,15 @@ typedef struct gm_plan_opts {
                               128-thread block each, symbolic then numeric pass over a compact array; larger
                               ones go to the dense W-column accumulator.  0 = default (4096 for fp32, 2048 for
                               fp64, less when shared memory is short), -1 = none                                 */
-  int32_t reserved[4];
+  int32_t expand_staging;  /* 1: the expansion that writes the first level's children brings the rows of B into
+                              shared memory with bulk asynchronous copies (one pipeline per warp; needs B's arrays
+                              16-byte aligned, otherwise ignored).  0 (default) / -1: ordinary loads, one tile of
+                              products per block — measured faster on B200 at every size tried               */
+  int32_t debug_spin_limit; /* testing aid: polls a kernel spends on a wait for bulk copies before it gives up and
+                              the call returns GM_ERR_TIMEOUT (0 = the default, about four million).  Negative:
+                              the copies are announced but withheld, so the wait runs out after that many polls
+                              with nothing in flight (how the tests reach the time-out path)                     */
+  int32_t reserved[2];
 } gm_plan_opts;
 
 /* What the host planner derives from (C.m, value size, smem_bytes): Section III-D. */

@@ -44,7 +44,8 @@ class PlanOpts(ctypes.Structure):
                 ("c_capacity", ctypes.c_int64), ("separate_histogram", ctypes.c_int32),
                 ("validate_inputs", ctypes.c_int32), ("single_stream", ctypes.c_int32),
                 ("level0_multisplit", ctypes.c_int32), ("small_chunk_max", ctypes.c_int32),
-                ("mid_chunk_max", ctypes.c_int32), ("reserved", ctypes.c_int32 * 4)]
+                ("mid_chunk_max", ctypes.c_int32), ("expand_staging", ctypes.c_int32),
+                ("debug_spin_limit", ctypes.c_int32), ("reserved", ctypes.c_int32 * 2)]
 
 
 class Params(ctypes.Structure):

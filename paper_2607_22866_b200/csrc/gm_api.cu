@@ -14,6 +14,7 @@
 #include "gm_k3_light.cuh"
 #include "gm_k4_expand.cuh"
 #include "gm_k4_direct.cuh"
+#include "gm_k4_stream.cuh"
 #include "gm_k5_multisplit.cuh"
 #include "gm_k6_accumulate.cuh"
 #include "gm_k7_gather.cuh"
@@ -165,6 +166,9 @@ struct gm_plan {
   uint32_t* seg_h = nullptr;       // H: segments of a batch x F0 (G minus the child boundary of the segment's row of B)
   uint32_t* seg_tile_sums = nullptr;
   bool direct = false;             // the expansion writes the level-0 children itself
+  bool stream = false;             // ... with the rows of B brought in by bulk copies (needs 16-byte aligned B arrays)
+  int32_t* seg_hrow = nullptr;     // n_seg: heavy row (position in the heavy-row list) of every segment
+  uint32_t* seg_rec = nullptr;     // segment records of a batch for the bulk-copy expansion (run starts + entry of A)
   int small_max = 0, mid_max = 0;  // size classes of the final chunks: <= small_max one warp, <= mid_max one small block
   std::vector<int64_t> heavy_nz_off_host;
   int64_t* heavy_nz_off = nullptr; // nH + 1
@@ -366,13 +370,14 @@ static int build_plan(gm_plan* p, cudaStream_t st) {
     GM_TRY(plan_alloc(p, &p->seg_bstart, static_cast<size_t>(p->n_seg) + 1, st));
     GM_TRY(plan_alloc(p, &p->seg_j, static_cast<size_t>(p->n_seg) + 1, st));
     GM_TRY(plan_alloc(p, &p->seg_brow, static_cast<size_t>(p->n_seg) + 1, st));
+    GM_TRY(plan_alloc(p, &p->seg_hrow, static_cast<size_t>(p->n_seg) + 1, st));
     k1_heavy_scatter<<<grid_for(nA, 256, p->num_sms), 256, 0, st>>>(p->heavy_flag, heavy_pos, p->ip, A.row_ptr, nA,
                                                                    p->x_heavy, heavy_ip, heavy_nnz);
     exclusive_scan<i64, i64>(heavy_ip, p->heavy_base, nH, p->scan_tmp, nullptr, nullptr, nullptr, st);
     exclusive_scan<i64, i64>(heavy_nnz, p->heavy_nz_off, nH, p->scan_tmp, nullptr, nullptr, nullptr, st);
     k1_heavy_segments<<<grid_for(p->n_seg + 1, 256, p->num_sms, 32), 256, 0, st>>>(
         p->x_heavy, nH, p->heavy_nz_off, p->heavy_base, A.row_ptr, A.col_idx, p->nz_off, B.row_ptr, p->n_seg, p->seg_off,
-        p->seg_bstart, p->seg_j, p->seg_brow);
+        p->seg_bstart, p->seg_j, p->seg_brow, p->seg_hrow);
     info.launches += 8;
     std::vector<int64_t> hb(static_cast<size_t>(nH) + 1);
     p->x_heavy_host.resize(static_cast<size_t>(nH));
@@ -398,6 +403,11 @@ static int build_plan(gm_plan* p, cudaStream_t st) {
     p->direct = prm.n_levels > 0 && prm.fanout[0] <= 256 &&
                 (p->opts.level0_multisplit == 2 || (p->opts.level0_multisplit == 0 && long_segments && bounds_fit));
     info.level0_direct = p->direct ? 1 : 0;
+    {
+      const size_t warp_smem = stream_warp_smem_bytes(prm.n_levels > 0 ? prm.fanout[0] : 2, p->sv);
+      p->stream = p->direct && p->opts.expand_staging == 1 && reinterpret_cast<uintptr_t>(B.col_idx) % 16 == 0 &&
+                  reinterpret_cast<uintptr_t>(B.vals) % 16 == 0 && p->smem_bytes >= kStreamWarps * warp_smem + 1024;
+    }
     // one staging buffer is enough when no multisplit pass runs (no levels, or one level done by the expansion)
     const int n_buf = prm.n_levels > (p->direct ? 1 : 0) ? 2 : 1;
 
@@ -457,6 +467,8 @@ static int build_plan(gm_plan* p, cudaStream_t st) {
       GM_TRY(plan_alloc(p, &p->seg_prefix, (static_cast<size_t>(max_seg_b) + 1) * static_cast<size_t>(F0), st));
       GM_TRY(plan_alloc(p, &p->seg_h, (static_cast<size_t>(max_seg_b) + 1) * static_cast<size_t>(F0), st));
       GM_TRY(plan_alloc(p, &p->seg_tile_sums, (static_cast<size_t>(max_seg_b) / kGTile + 2) * static_cast<size_t>(F0), st));
+      if (p->stream)
+        GM_TRY(plan_alloc(p, &p->seg_rec, (static_cast<size_t>(max_seg_b) + 1) * static_cast<size_t>(stream_rec_words(F0)), st));
       if (B.n_rows > 0) {
         k_child_bounds<<<grid_for(B.n_rows * (F0 + 1), 256, p->num_sms, 32), 256, 0, st>>>(B.row_ptr, B.col_idx, B.n_rows, F0,
                                                                                         prm.shift[0], p->child_bound);
@@ -658,14 +670,38 @@ static int heavy_batch_front(gm_plan* p, const Batch& b, HeavyBatchState<V>* hs,
     p->stats.launches += 4;
     tm.end(st);
     tm.begin(PhaseTimes::kExpand, st);
-    const unsigned grid = static_cast<unsigned>((b.elems + kExpandTile - 1) / kExpandTile);
-    k_tile_bounds<<<grid_for(grid, 256, p->num_sms), 256, 0, st>>>(p->seg_off, p->n_seg, b.elem0, b.elems, kExpandTile,
-                                                                 p->tile_meta);
-    k_tile_bounds<<<grid_for(grid, 256, p->num_sms), 256, 0, st>>>(off_cur, rows_b, 0, b.elems, kExpandTile, p->row_meta);
-    k4_expand_direct<V><<<grid, kExpandThreads, 0, st>>>(
-        p->seg_off, p->seg_bstart, p->seg_j, p->tile_meta, static_cast<const V*>(p->A.vals), p->B.col_idx,
-        static_cast<const V*>(p->B.vals), b.elem0, b.elems, p->row_meta, off_cur, seg0, F, prm.shift[0], row_base, p->seg_h,
-        p->stage_col[0], static_cast<V*>(p->stage_val[0]));
+    if (p->stream) {
+      // one contiguous range of the batch's products per warp; the grid fills the SMs' shared memory
+      const size_t smem = kStreamWarps * stream_warp_smem_bytes(F, sizeof(V));
+      const int per_sm = std::max<int>(1, std::min<int>(16, static_cast<int>((p->smem_bytes - 1024) / (smem + 1024))));
+      const i64 n_warps = static_cast<i64>(p->num_sms) * per_sm * kStreamWarps;
+      const i64 per_warp = std::max<i64>(4096, ((b.elems + n_warps - 1) / n_warps + 127) & ~i64{127});
+      const i64 n_ranges = (b.elems + per_warp - 1) / per_warp;
+      const unsigned grid = static_cast<unsigned>((n_ranges + kStreamWarps - 1) / kStreamWarps);
+      k_seg_records<V><<<grid_for(n_seg_b * stream_rec_words(F), 256, p->num_sms, 32), 256, 0, st>>>(
+          p->seg_h, row_base, p->seg_hrow, p->seg_j, static_cast<const V*>(p->A.vals), seg0, n_seg_b, b.h0, F, p->seg_rec);
+      k_tile_bounds<<<grid_for(n_ranges, 256, p->num_sms), 256, 0, st>>>(p->seg_off, p->n_seg, b.elem0, b.elems,
+                                                                       static_cast<int>(per_warp), p->tile_meta);
+      auto kern = k4_expand_stream<V>;
+      GM_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)));
+      const int spin = p->opts.debug_spin_limit != 0 ? p->opts.debug_spin_limit : kCopySpinLimit;
+      kern<<<grid, kStreamWarps * 32, smem, st>>>(p->seg_off, p->seg_bstart, p->n_seg, p->tile_meta, p->B.col_idx,
+                                                  static_cast<const V*>(p->B.vals), p->B.nnz, b.elem0, b.elems, per_warp, seg0,
+                                                  p->seg_rec, F, prm.shift[0], p->stage_col[0], static_cast<V*>(p->stage_val[0]),
+                                                  spin, p->err);
+      k4_expand_short<V><<<grid_for(n_seg_b * 32, 256, p->num_sms, 8), 256, 0, st>>>(
+          p->seg_off, p->seg_bstart, p->B.col_idx, static_cast<const V*>(p->B.vals), seg0, n_seg_b, p->seg_rec, F, prm.shift[0],
+          p->stage_col[0], static_cast<V*>(p->stage_val[0]));
+    } else {
+      const unsigned grid = static_cast<unsigned>((b.elems + kExpandTile - 1) / kExpandTile);
+      k_tile_bounds<<<grid_for(grid, 256, p->num_sms), 256, 0, st>>>(p->seg_off, p->n_seg, b.elem0, b.elems, kExpandTile,
+                                                                   p->tile_meta);
+      k_tile_bounds<<<grid_for(grid, 256, p->num_sms), 256, 0, st>>>(off_cur, rows_b, 0, b.elems, kExpandTile, p->row_meta);
+      k4_expand_direct<V><<<grid, kExpandThreads, 0, st>>>(
+          p->seg_off, p->seg_bstart, p->seg_j, p->tile_meta, static_cast<const V*>(p->A.vals), p->B.col_idx,
+          static_cast<const V*>(p->B.vals), b.elem0, b.elems, p->row_meta, off_cur, seg0, F, prm.shift[0], row_base, p->seg_h,
+          p->stage_col[0], static_cast<V*>(p->stage_val[0]));
+    }
     p->stats.launches += 3;
     GM_CUDA(cudaGetLastError());
     tm.end(st);

@@ -80,6 +80,44 @@ __device__ __forceinline__ int clamp_rel(i64 v, int lo, int hi) {
   return v < lo ? lo : (v > hi ? hi : static_cast<int>(v));
 }
 
+// ---- asynchronous bulk copies into shared memory (cp.async.bulk + mbarrier), this block's own memory only
+__device__ __forceinline__ u32 smem_u32(const void* p) { return static_cast<u32>(__cvta_generic_to_shared(p)); }
+
+__device__ __forceinline__ void mbar_init(u64* bar, int count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_fence_init() { asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory"); }
+// one arrival that also announces `bytes` of copies (0: a plain arrival)
+__device__ __forceinline__ void mbar_arrive_expect_tx(u64* bar, u32 bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(u64* bar, u32 parity) {
+  u32 ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(smem_u32(bar)), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+// 1-D bulk copy global -> this block's shared memory; both addresses 16-byte aligned, bytes a multiple of 16
+__device__ __forceinline__ void bulk_g2s(void* dst, const void* src, u32 bytes, u64* bar) {
+  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(smem_u32(dst)),
+               "l"(src), "r"(bytes), "r"(smem_u32(bar))
+               : "memory");
+}
+// Bounded wait: polls with back-off at most `limit` times; false = gave up (the caller records kDevTimeout).
+__device__ __forceinline__ bool mbar_wait_bounded(u64* bar, u32 parity, int limit) {
+  for (int spins = 0; spins < limit; ++spins) {
+    if (mbar_try_wait(bar, parity)) return true;
+    __nanosleep(64);
+  }
+  return mbar_try_wait(bar, parity);
+}
+constexpr int kCopySpinLimit = 1 << 22;  // default number of polls before a wait on bulk copies gives up
+
 // What a tile-per-block kernel needs to know about the groups (rows, parents, segments) its tile touches.
 struct __align__(16) TileMeta {
   i64 first;  // group that contains the tile's first element

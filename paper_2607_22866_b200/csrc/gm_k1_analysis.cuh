@@ -98,7 +98,7 @@ __global__ void k1_heavy_segments(const int32_t* __restrict__ x_heavy, i64 n_hea
                                   const int32_t* __restrict__ a_col, const i64* __restrict__ nz_off,
                                   const i64* __restrict__ b_row_ptr, i64 n_seg, i64* __restrict__ seg_off,
                                   i64* __restrict__ seg_bstart, i64* __restrict__ seg_j,
-                                  int32_t* __restrict__ seg_brow) {
+                                  int32_t* __restrict__ seg_brow, int32_t* __restrict__ seg_hrow) {
   for (i64 s = static_cast<i64>(blockIdx.x) * blockDim.x + threadIdx.x; s <= n_seg;
        s += static_cast<i64>(gridDim.x) * blockDim.x) {
     if (s == n_seg) { seg_off[s] = heavy_base[n_heavy]; continue; }
@@ -110,6 +110,7 @@ __global__ void k1_heavy_segments(const int32_t* __restrict__ x_heavy, i64 n_hea
     seg_bstart[s] = b_row_ptr[a_col[j]];
     seg_j[s] = j;
     seg_brow[s] = a_col[j];
+    seg_hrow[s] = static_cast<int32_t>(h);
   }
 }
 

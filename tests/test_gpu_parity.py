@@ -350,6 +350,32 @@ def test_expansion_straight_into_the_first_level(dtype, fanout, width):
     assert info.level0_direct == 1 and info.n_batches > 1 and info.params.n_levels >= 1
 
 
+@pytest.mark.parametrize("dtype,fanout,width", [(np.float32, 32, 512), (np.float64, 128, 128), (np.float32, 2, 8192)])
+def test_bulk_copy_expansion_and_plain_loads_agree(dtype, fanout, width):
+    # expand_staging = 1: rows of B reach the expansion through bulk asynchronous copies into shared memory (pieces
+    # that start and end at every alignment, warps whose range holds one segment or hundreds, short segments by the
+    # kernel of their own, the last elements of B's arrays); default: the tile-per-block kernel with plain loads.
+    # Both against the oracle.
+    A = gen.rmat(14, 16, seed=13, dtype=dtype)
+    kw = dict(tau=512, chunk_width=width, max_fanout=fanout, stage_elems=1 << 22, level0_multisplit=2)
+    C1, info, _ = check_product(A, A, expand_staging=1, **kw)
+    assert info.level0_direct == 1 and info.n_batches > 1 and info.params.levels()[0] == fanout
+    C2, info2, _ = check_product(A, A, **kw)
+    assert torch.equal(C1.row_ptr, C2.row_ptr) and torch.equal(C1.col, C2.col)
+
+
+def test_bounded_wait_on_bulk_copies_runs_out_cleanly():
+    # the copies are announced to the barrier but withheld (nothing completes it), so every wait gives up after 200
+    # polls: the call returns GM_ERR_TIMEOUT, nothing faults or hangs, and the same context then computes the product
+    import paper_2607_22866_b200 as gm
+    A = gen.rmat(13, 16, seed=13, dtype=np.float32)
+    kw = dict(tau=512, chunk_width=1024, max_fanout=8, level0_multisplit=2)
+    with pytest.raises(gm.GmError) as ei:
+        run_gpu(A, A, expand_staging=1, debug_spin_limit=-200, **kw)
+    assert ei.value.status == -8
+    check_product(A, A, expand_staging=1, **kw)
+
+
 def test_expansion_straight_into_the_first_level_short_rows_of_b():
     # rows of B with 0 to 3 entries: tiles with thousands of segments, empty segments, heavy rows made of them
     rng = np.random.default_rng(23)
