@@ -3,6 +3,7 @@ checks.  This package holds no SpGEMM arithmetic: it only builds CSR inputs."""
 from .matrices import (  # noqa: F401
     CSR,
     counter_uniform,
+    block_dense_rows,
     erdos_renyi_k,
     laplacian_2d,
     rmat,

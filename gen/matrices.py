@@ -19,6 +19,9 @@ rectangular pair stands in for its web/social-graph matrices):
                       duplicate edges merged before values are drawn.
 * ``zipf_rows``       row lengths min(X, cap) with P(X = k) proportional to k**-s (k >= 1),
                       columns uniform and distinct inside a row.
+* ``block_dense_rows`` block rows that couple to a handful of block columns with dense blocks (the shape of the
+                      paper's structural and power-network matrices, Table II: few thousand rows per pattern, most
+                      rows heavy, nearly every product in a heavy row, a narrow column space).
 """
 from __future__ import annotations
 
@@ -232,17 +235,64 @@ def zipf_rectangular_pair(n_a: int, m_a: int, m_b: int, seed: int, dtype=np.floa
     return A, B
 
 
+_STREAM_BLOCKS = 1 << 43
+
+
+def block_dense_rows(n: int, block: int, blocks_per_row: int, fill: float, dense_frac: float, seed: int,
+                     dtype=np.float32) -> CSR:
+    """Square matrix of ``n / block`` block rows shaped like the stiffness and power-network matrices whose
+    squares are almost all heavy rows (few thousand rows per block structure, rows of a few hundred entries in
+    dense blocks, a column space of a few accumulator widths).  A *dense* block row (probability ``dense_frac``)
+    couples to itself, its two neighbours and ``blocks_per_row - 3`` uniform-random block columns; inside a coupled
+    block every entry is kept with probability ``fill``.  The other block rows keep the diagonal and about two
+    more entries of their own diagonal block per row, so their rows stay light.  Duplicate block choices merge."""
+    assert n % block == 0 and blocks_per_row >= 3
+    nb = n // block
+    br = np.arange(nb, dtype=np.int64)
+    dense = counter_uniform(seed, _STREAM_BLOCKS, br) < dense_frac
+    # chosen block columns, (nb, blocks_per_row): self, neighbours (wrapping), random
+    choice = np.empty((nb, blocks_per_row), dtype=np.int64)
+    choice[:, 0] = br
+    choice[:, 1] = (br + 1) % nb
+    choice[:, 2] = (br + nb - 1) % nb
+    for j in range(3, blocks_per_row):
+        u = counter_uniform(seed, _STREAM_BLOCKS + j, br)
+        choice[:, j] = np.minimum((u * nb).astype(np.int64), nb - 1)
+    parts = []
+    db = br[dense]
+    for j in range(blocks_per_row):
+        # candidate entries of block (db, choice[db, j]): index = ((block row * blocks_per_row + j) * block + r) * block + c
+        r, c = np.meshgrid(np.arange(block, dtype=np.int64), np.arange(block, dtype=np.int64), indexing="ij")
+        base = ((db * blocks_per_row + j) * block)[:, None, None]
+        idx = (base + r[None]) * block + c[None]
+        keep = counter_uniform(seed, _STREAM_COLUMNS, idx.ravel()).reshape(idx.shape) < fill
+        rows = (db[:, None, None] * block + r[None])[keep]
+        cols = (choice[db, j][:, None, None] * block + c[None])[keep]
+        parts.append(rows * n + cols)
+    sb = br[~dense]
+    if sb.size:
+        r, c = np.meshgrid(np.arange(block, dtype=np.int64), np.arange(block, dtype=np.int64), indexing="ij")
+        idx = ((sb * blocks_per_row)[:, None, None] * block + r[None]) * block + c[None]
+        keep = (counter_uniform(seed, _STREAM_COLUMNS, idx.ravel()).reshape(idx.shape) < 2.0 / block) | (r == c)[None]
+        rows = (sb[:, None, None] * block + r[None])[keep]
+        cols = (sb[:, None, None] * block + c[None])[keep]
+        parts.append(rows * n + cols)
+    keys = np.unique(np.concatenate(parts))
+    return _csr_from_sorted_keys(keys, n, n, seed, dtype)
+
+
 CONFIG_NAMES = [
     "er4096_k8_f32",
     "laplacian1024_f64",
     "rmat20_ef16_f32",
     "rmat21_ef8_f64",
     "zipf_rect_f32",
+    "block_dense_f32",
 ]
 
 
 def config_inputs(index: int, shrink: int = 0):
-    """The five benchmark products.  ``shrink`` > 0 scales the problem down by 2**shrink (rows and
+    """The five benchmark products, and (index 5) a product of the second workload class.  ``shrink`` > 0 scales the problem down by 2**shrink (rows and
     columns; grid side for the Laplacian) with the same recipe, for tests the oracle finishes in
     seconds.  Returns (A, B, description)."""
     if index == 0:
@@ -266,4 +316,11 @@ def config_inputs(index: int, shrink: int = 0):
                                      seed=5, dtype=np.float32)
         return A, B, (f"C=A*B, A {A.n_rows}x{A.n_cols} Zipf(1.8) rows capped 4096, "
                       f"B {B.n_rows}x{B.n_cols} Zipf(2.0) rows capped 2048, fp32, seed 5")
-    raise ValueError(f"config index {index} out of range 0..4")
+    if index == 5:
+        # second workload class: dense-ish heavy rows, almost every product in a heavy row, a column space of two
+        # accumulator widths (one multisplit level, the chunk accumulation dominates)
+        n = 65536 >> shrink
+        A = block_dense_rows(n, 64, 6, 0.7, 0.7, seed=6, dtype=np.float32)
+        return A, A, (f"C=A*A, {n}x{n} in 64x64 blocks, 70% dense block rows coupling to 6 block columns at fill 0.7, "
+                      f"fp32, seed 6")
+    raise ValueError(f"config index {index} out of range 0..5")

@@ -73,8 +73,12 @@ typedef struct gm_plan_opts {
   int64_t c_capacity;      /* room, in entries, reserved for C when heavy rows need > 1 batch  */
   int32_t separate_histogram; /* 1: always run the stand-alone histogram kernel per level (otherwise a
                               first level that runs as separate passes is counted by the expansion) */
-  int32_t validate_inputs; /* 1: check row_ptr / col_idx of A and B on the device first        */
-  int32_t single_stream;   /* accepted and ignored: all work of a call runs on the caller's stream */
+  int32_t validate_inputs; /* 1: debug mode.  row_ptr / col_idx of A and B are checked on the device first
+                              (GM_ERR_BAD_CSR), and before every chunk accumulation a pass over the staging buffer
+                              checks that each product lies in the columns its chunk owns (GM_ERR_INTERNAL)     */
+  int32_t single_stream;   /* 1: every kernel of a call runs on the caller's stream.  0 (default): the light rows'
+                              kernels run on a second stream of the plan's, forked from and joined back into the
+                              caller's stream with events, next to the heavy rows' kernels (Algorithm 3)      */
   int32_t level0_multisplit; /* first multisplit level: 1 = separate histogram and multisplit passes over
                               the staging buffer (Algorithm 5 as printed); 2 = the expansion kernel writes
                               the first level's children itself; 0 (default) = the latter when the heavy
@@ -200,8 +204,9 @@ int gm_spgemm_plan_ex(const gm_csr* A, const gm_csr* B, size_t smem_bytes,
  * C.row_ptr is known by prefix sums over the per-row counts, the gather of the chunks into C.
  *   C_out  host struct filled with device pointers allocated through the allocator hook;
  *          C_out->nnz is exact.  Release with gm_csr_free.
- * Work is enqueued on `cuda_stream`; the call returns after synchronising that stream, because nnz(C)
- * is needed on the host.
+ * Work is enqueued on `cuda_stream` (the light rows' kernels on a second stream ordered inside it by events,
+ * unless single_stream is set); the call returns after synchronising that stream, because nnz(C) is needed
+ * on the host.
  * A plan can be executed any number of times (values of A and B may change in between, their
  * structure may not).  Two executes of the same plan must not overlap.
  * Errors: GM_ERR_CAPACITY (C did not fit the reserved room; only possible when the heavy rows

@@ -197,6 +197,9 @@ struct gm_plan {
   gm::TileMeta* tile_meta = nullptr;  // per tile of the expansion / multisplit kernels: groups it touches
   gm::PhaseTimes times;
   HostSink* sink = nullptr;        // set by gm_spgemm_host for the duration of one execute
+  // light rows run next to the heavy path on a stream of the plan's own (Algorithm 3 keeps separate queues for them)
+  cudaStream_t light_stream = nullptr;
+  cudaEvent_t ev_fork = nullptr, ev_light = nullptr;
 };
 
 namespace gm {
@@ -564,6 +567,11 @@ static int launch_accumulate(gm_plan* p, const Batch& b, const HeavyBatchState<V
   const int small_max = p->small_max, mid_max = p->mid_max;
   GM_CUDA(cudaMemsetAsync(p->acc_counters, 0, 8 * sizeof(int), st));
   GM_CUDA(cudaMemsetAsync(p->chunk_nnz, 0, static_cast<size_t>(hs.n_chunks) * sizeof(u32), st));
+  if (p->opts.validate_inputs) {
+    k6_validate_chunks<<<grid_for(hs.n_chunks * 32, 256, p->num_sms, 8), 256, 0, st>>>(hs.fin_col, hs.chunk_off, hs.n_chunks,
+                                                                                      hs.log2_cpr, W, p->B.n_cols, p->err);
+    ++p->stats.launches;
+  }
   k6_classify<<<grid_for(hs.n_chunks, 256, p->num_sms), 256, 0, st>>>(hs.chunk_off, hs.n_chunks, small_max, mid_max, p->mid_list,
                                                                      p->big_list, p->acc_counters);
   ++p->stats.launches;
@@ -820,7 +828,35 @@ static int execute_t(gm_plan* p, cudaStream_t st, gm_csr* C) {
   if (!c_row_ptr) return fail(GM_ERR_OOM, "allocation of C.row_ptr failed");
   int32_t* c_col = nullptr;
   V* c_val = nullptr;
+  // ---- light and heavy rows are independent until C.row_ptr is formed: the light rows' kernels go to a second
+  // stream, forked from and joined back into the caller's with events (never when single_stream is set)
+  bool fork = !p->opts.single_stream && info.rows_light > 0 && info.rows_heavy > 0;
+  if (fork && !p->light_stream) {
+    // one second stream per device for the life of the process (creating and destroying a stream per plan cost more
+    // than the overlap gained on millisecond products); executes that share it are ordered by their own events
+    static cudaStream_t side_streams[64] = {nullptr};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) {
+      fork = false;
+    } else {
+      if (!side_streams[dev] && cudaStreamCreateWithFlags(&side_streams[dev], cudaStreamNonBlocking) != cudaSuccess) {
+        cudaGetLastError();
+        side_streams[dev] = nullptr;
+      }
+      p->light_stream = side_streams[dev];
+      if (!p->light_stream || cudaEventCreateWithFlags(&p->ev_fork, cudaEventDisableTiming) != cudaSuccess ||
+          cudaEventCreateWithFlags(&p->ev_light, cudaEventDisableTiming) != cudaSuccess) {
+        cudaGetLastError();
+        p->light_stream = nullptr;
+        fork = false;
+      }
+    }
+  }
+  cudaStream_t lst = fork ? p->light_stream : st;
+  auto fork_light = [&]() { if (fork) { cudaEventRecord(p->ev_fork, st); cudaStreamWaitEvent(lst, p->ev_fork, 0); } };
+  auto join_light = [&]() { if (fork) { cudaEventRecord(p->ev_light, lst); cudaStreamWaitEvent(st, p->ev_light, 0); } };
   auto cleanup = [&]() {
+    if (fork) cudaStreamSynchronize(lst);
     if (p->sink && p->sink->copy_stream) cudaStreamSynchronize(p->sink->copy_stream);  // copies out of C in flight
     dev_free(c_row_ptr, st);
     dev_free(c_col, st);
@@ -829,9 +865,11 @@ static int execute_t(gm_plan* p, cudaStream_t st, gm_csr* C) {
 #define GM_TRY_C(expr) do { int rc2_ = (expr); if (rc2_ != GM_OK) { cudaStreamSynchronize(st); cleanup(); return rc2_; } } while (0)
 
   // ---- light rows, symbolic (Algorithm 3: Symbolic(A[x_light,:], B))
-  tm.begin(PhaseTimes::kLightSym, st);
-  GM_TRY_C((launch_light<V, false>(p, p->sym_rows, p->sym_fill, info.light_bin_rows, nullptr, nullptr, nullptr, 0, st)));
-  tm.end(st);
+  fork_light();
+  tm.begin(PhaseTimes::kLightSym, lst);
+  GM_TRY_C((launch_light<V, false>(p, p->sym_rows, p->sym_fill, info.light_bin_rows, nullptr, nullptr, nullptr, 0, lst)));
+  tm.end(lst);
+  bool light_counted = !fork;  // the heavy path joins before the first prefix sum over the per-row counts
 
   // a row's numeric bin is never above its symbolic bin
   i64 num_upper[kMaxLightBins] = {0};
@@ -840,19 +878,19 @@ static int execute_t(gm_plan* p, cudaStream_t st, gm_csr* C) {
     for (int b = p->bins.n_bins - 1; b >= 0; --b) { run += info.light_bin_rows[b]; num_upper[b] = run; }
   }
   // numeric pass of the light rows in [r0, r1) (all of them by default)
-  auto light_numeric_range = [&](i64 capacity, i64 r0, i64 r1) -> int {
-    tm.begin(PhaseTimes::kLightNum, st);
+  auto light_numeric_range = [&](i64 capacity, i64 r0, i64 r1, cudaStream_t s2) -> int {
+    tm.begin(PhaseTimes::kLightNum, s2);
     if (info.rows_light > 0 && r1 > r0) {
-      GM_CUDA(cudaMemsetAsync(p->num_fill, 0, 8 * sizeof(int), st));
-      k1_bin_rows<int32_t><<<static_cast<unsigned>((r1 - r0 + 255) / 256), 256, 0, st>>>(
+      GM_CUDA(cudaMemsetAsync(p->num_fill, 0, 8 * sizeof(int), s2));
+      k1_bin_rows<int32_t><<<static_cast<unsigned>((r1 - r0 + 255) / 256), 256, 0, s2>>>(
           p->row_nnz + r0, p->heavy_flag + r0, r1 - r0, p->bins, std::max<i64>(nA, 1), p->num_fill, p->num_rows, r0);
       ++p->stats.launches;
-      GM_TRY((launch_light<V, true>(p, p->num_rows, p->num_fill, num_upper, c_row_ptr, c_col, c_val, capacity, st)));
+      GM_TRY((launch_light<V, true>(p, p->num_rows, p->num_fill, num_upper, c_row_ptr, c_col, c_val, capacity, s2)));
     }
-    tm.end(st);
+    tm.end(s2);
     return GM_OK;
   };
-  auto light_numeric = [&](i64 capacity) -> int { return light_numeric_range(capacity, 0, nA); };
+  auto light_numeric = [&](i64 capacity, cudaStream_t s2) -> int { return light_numeric_range(capacity, 0, nA, s2); };
 
   const size_t n_batches = p->batches.size();
   i64 capacity = 0;
@@ -863,6 +901,8 @@ static int execute_t(gm_plan* p, cudaStream_t st, gm_csr* C) {
     // ---- everything is resident at once: count, allocate C exactly, then fill
     HeavyBatchState<V> hs;
     if (n_batches == 1) GM_TRY_C(heavy_batch_front<V>(p, p->batches[0], &hs, st));
+    join_light();
+    light_counted = true;
     tm.begin(PhaseTimes::kScan, st);
     exclusive_scan<int32_t, i64>(p->row_nnz, c_row_ptr, nA, p->scan_tmp, nullptr, p->c_total, nullptr, st);
     p->stats.launches += 3;
@@ -876,12 +916,15 @@ static int execute_t(gm_plan* p, cudaStream_t st, gm_csr* C) {
     c_col = static_cast<int32_t*>(dev_alloc(static_cast<size_t>(std::max<i64>(total, 1)) * sizeof(int32_t), st));
     c_val = static_cast<V*>(dev_alloc(static_cast<size_t>(std::max<i64>(total, 1)) * sizeof(V), st));
     if (!c_col || !c_val) { cleanup(); return fail(GM_ERR_OOM, "allocation of C (" + std::to_string(total) + " entries) failed"); }
+    // the gather of the heavy rows and the numeric pass of the light rows write different rows of C
+    fork_light();
     if (n_batches == 1) {
       tm.begin(PhaseTimes::kAccSym, st);
       GM_TRY_C((launch_gather<V>(p, p->batches[0], hs, c_row_ptr, c_col, c_val, capacity, st)));
       tm.end(st);
     }
-    GM_TRY_C(light_numeric(capacity));
+    GM_TRY_C(light_numeric(capacity, lst));
+    join_light();
   } else {
     // ---- heavy rows in several staging-buffer fills: C is appended in row order into reserved room
     // Room for C.  Given: use it.  Derived: the structural upper bound sum_i min(IP_i, C.m), cut
@@ -916,6 +959,7 @@ static int execute_t(gm_plan* p, cudaStream_t st, gm_csr* C) {
       const Batch& b = p->batches[bi];
       HeavyBatchState<V> hs;
       GM_TRY_C(heavy_batch_front<V>(p, b, &hs, st));
+      if (!light_counted) { join_light(); light_counted = true; }
       // rows [r0, r1) of C get their offsets now: every light row in the range was counted up front
       const i64 r0 = bi == 0 ? 0 : p->x_heavy_host[static_cast<size_t>(b.h0)];
       const i64 r1 = bi + 1 == n_batches ? nA : p->x_heavy_host[static_cast<size_t>(p->batches[bi + 1].h0)];
@@ -929,7 +973,7 @@ static int execute_t(gm_plan* p, cudaStream_t st, gm_csr* C) {
       if (HostSink* sk = p->sink) {
         // The caller wants C on the host: finish rows [r0, r1) now (their light rows too), note how many entries
         // of C that makes, and send the previous batch's entries on their way while this batch computes.
-        GM_TRY_C(light_numeric_range(capacity, r0, r1));
+        GM_TRY_C(light_numeric_range(capacity, r0, r1, st));
         if (sk->events.size() <= bi) {
           cudaEvent_t ev = nullptr;
           if (cudaEventCreateWithFlags(&ev, cudaEventDisableTiming) != cudaSuccess) { cleanup(); return fail(GM_ERR_CUDA, "event creation failed"); }
@@ -953,7 +997,7 @@ static int execute_t(gm_plan* p, cudaStream_t st, gm_csr* C) {
         if (bi + 1 == n_batches) send(bi);
       }
     }
-    if (!p->sink) GM_TRY_C(light_numeric(capacity));
+    if (!p->sink) GM_TRY_C(light_numeric(capacity, st));
     if (cudaMemcpyAsync(&total, p->c_total, sizeof(i64), cudaMemcpyDeviceToHost, st) != cudaSuccess) {
       cleanup();
       return fail(GM_ERR_CUDA, "copy of nnz(C) failed");
@@ -1105,6 +1149,8 @@ void gm_csr_free(gm_csr* C) {
 
 void gm_plan_destroy(gm_plan* plan) {
   if (!plan) return;
+  if (plan->ev_fork) cudaEventDestroy(plan->ev_fork);
+  if (plan->ev_light) cudaEventDestroy(plan->ev_light);
   for (auto& b : plan->owned) dev_free(b.p, plan->plan_stream);
   delete plan;
 }

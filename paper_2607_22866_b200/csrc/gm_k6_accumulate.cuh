@@ -67,6 +67,26 @@ __global__ void k6_classify(const i64* __restrict__ chunk_off, i64 n_chunks, int
   }
 }
 
+// Debug net (plan option validate_inputs): every product that reaches the accumulate kernels must lie in the W
+// columns its chunk owns.  One warp per chunk; a violation sets kDevBadChunk (the kernels themselves mask the
+// column and would fold a misplaced product into the wrong entry silently).
+__global__ void k6_validate_chunks(const int32_t* __restrict__ x_col, const i64* __restrict__ chunk_off, i64 n_chunks,
+                                   int log2_chunks_per_row, int W, i64 n_cols, int* __restrict__ err) {
+  const int lane = threadIdx.x & 31;
+  const int log2W = 31 - __clz(W);
+  const u32 crow_mask = (1u << log2_chunks_per_row) - 1u;
+  const i64 n_warps = static_cast<i64>(gridDim.x) * (blockDim.x >> 5);
+  for (i64 k = static_cast<i64>(blockIdx.x) * (blockDim.x >> 5) + (threadIdx.x >> 5); k < n_chunks; k += n_warps) {
+    const u32 want = static_cast<u32>(k) & crow_mask;
+    bool bad = false;
+    for (i64 q = chunk_off[k] + lane; q < chunk_off[k + 1]; q += 32) {
+      const int32_t c = x_col[q];
+      bad |= c < 0 || c >= n_cols || (static_cast<u32>(c) >> log2W) != want;
+    }
+    if (bad) dev_set_error(err, kDevBadChunk);
+  }
+}
+
 // Position in C of every chunk's first entry, once C.rowPtr of the batch's rows is known.
 __global__ void k6_chunk_bases(const i64* __restrict__ chunk_nnz_off, i64 n_chunks, int log2_chunks_per_row,
                                const int32_t* __restrict__ x_heavy, i64 h0, const i64* __restrict__ c_row_ptr,

@@ -58,3 +58,17 @@ def test_zipf_lengths_follow_the_clipped_law():
     assert abs((lens == 2).mean() - p1 * 2 ** -1.8) < 0.01
     tail = 1.0 - np.sum(np.arange(1, 4096, dtype=np.float64) ** -1.8) / zeta(1.8)
     assert abs((lens == 4096).mean() - tail) < 5e-4 and (lens == 4096).sum() > 0
+
+
+def test_block_dense_rows_is_the_second_workload_class():
+    # most rows heavy, nearly every product in a heavy row, column space of a few accumulator widths
+    import oracle
+    A, B, _ = gen.config_inputs(5, shrink=4)
+    A.validate()
+    assert B is A and A.n_rows == A.n_cols == 4096
+    A2, _, _ = gen.config_inputs(5, shrink=4)
+    assert np.array_equal(A.col, A2.col) and np.array_equal(A.val, A2.val)   # same seed, same matrix
+    ip = oracle.row_products(A, A)
+    heavy = ip > 512
+    assert 0.3 <= heavy.mean() <= 0.9 and ip[heavy].sum() >= 0.98 * ip.sum()
+    assert np.diff(A.row_ptr).min() >= 1 and np.diff(A.row_ptr).max() <= 6 * 64

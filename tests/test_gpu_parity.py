@@ -175,6 +175,21 @@ def test_argument_errors():
     assert ei.value.status == -4
 
 
+@pytest.mark.parametrize("dtype", [np.float32, np.float64])
+def test_single_stream_and_debug_validation(dtype):
+    # light rows next to the heavy path on the plan's second stream (default) or everything on the caller's stream;
+    # debug mode checks the inputs and every product's chunk on the device and finds nothing to complain about
+    A = gen.rmat(13, 16, seed=4, dtype=dtype)
+    kw = dict(tau=256, chunk_width=1024, max_fanout=4, stage_elems=1 << 21)
+    C1, info, _ = check_product(A, A, **kw)
+    assert info.rows_light > 0 and info.rows_heavy > 0 and info.n_batches > 1 and info.params.n_levels == 2
+    C2, _, _ = check_product(A, A, single_stream=1, validate_inputs=1, **kw)
+    assert torch.equal(C1.row_ptr, C2.row_ptr) and torch.equal(C1.col, C2.col)
+    A1, B1, _ = gen.config_inputs(4, shrink=6)      # one batch: gather and the light rows' numeric pass side by side
+    check_product(A1, B1, validate_inputs=1)
+    check_product(A1, B1, single_stream=1)
+
+
 def test_two_runs_same_structure_values_close():
     A = gen.rmat(12, 16, seed=9, dtype=np.float32)
     C1, _, _ = run_gpu(A, A, tau=256, chunk_width=1024, max_fanout=4)
@@ -302,6 +317,19 @@ def test_config4_zipf_pair_full_size_default_plan():
     A, B, _ = gen.config_inputs(4)
     info, stats = _check_sampled_rows(A, B, n_random=150, n_heavy=60, whole_row_ptr=True)
     assert info.params.levels() == [256, 2] and info.level0_direct == 0 and info.rows_heavy > 0
+
+
+def test_second_workload_class_dense_heavy_rows():
+    # block-structured product (the shape of the paper's structural matrices): 70 % of the rows heavy, 99.99 % of the
+    # products in them, two chunks per row, rows of C of a thousand entries from tens of thousands of products.
+    # Whole matrix against the oracle at 1/16 size, sampled rows and every row's entry count at full size.
+    A, B, _ = gen.config_inputs(5, shrink=4)
+    C, info, stats = check_product(A, B)
+    assert info.rows_heavy > 0.5 * A.n_rows
+    A, B, _ = gen.config_inputs(5)
+    info, stats = _check_sampled_rows(A, B, n_random=100, n_heavy=60, whole_row_ptr=True)
+    assert info.params.levels() == [2] and info.products_heavy > 0.98 * info.products_total
+    assert stats.c_nnz * 20 < info.products_total   # dense accumulation: dozens of products per entry
 
 
 def test_config3_rmat_fp64_two_levels_sampled_rows():
