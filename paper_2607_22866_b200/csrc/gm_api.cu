@@ -276,7 +276,7 @@ static int build_plan(gm_plan* p, cudaStream_t st) {
     const gm_plan_opts& o = p->opts;
     if (o.small_chunk_max < -1 || o.small_chunk_max > kAccSmallChunk || o.mid_chunk_max < -1 || o.mid_chunk_max > (1 << 15))
       return fail(GM_ERR_INVALID_ARG, "small_chunk_max / mid_chunk_max out of range");
-    p->small_max = o.small_chunk_max < 0 ? 0 : (o.small_chunk_max ? o.small_chunk_max : kAccSmallChunk);
+    p->small_max = o.small_chunk_max < 0 ? 0 : (o.small_chunk_max ? o.small_chunk_max : kAccSmallDefault);
     int mid = o.mid_chunk_max < 0 ? 0 : (o.mid_chunk_max ? o.mid_chunk_max : (p->sv == 4 ? 4096 : 2048));
     // several mid-chunk blocks must fit an SM next to each other for the class to pay
     while (mid > p->small_max && mid_smem_bytes(prm.chunk_width, p->sv, mid) + 1024 > p->smem_bytes / 8) mid /= 2;
@@ -746,6 +746,7 @@ static int heavy_batch_front(gm_plan* p, const Batch& b, HeavyBatchState<V>* hs,
     GM_CUDA(cudaFuncSetAttribute(k5_level<V, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                  static_cast<int>(split_smem_bytes<V>(true))));
   }
+  bool hist_ready = false;  // the previous level's multisplit counted this level's bins while it wrote
   for (int l = first_level; l < prm.n_levels; ++l) {
     const int F = prm.fanout[l];
     const i64 n_child = n_par * F;
@@ -755,10 +756,10 @@ static int heavy_batch_front(gm_plan* p, const Batch& b, HeavyBatchState<V>* hs,
     tm.begin(PhaseTimes::kHist, st);
     k_tile_bounds<<<grid_for(grid, 256, p->num_sms), 256, 0, st>>>(off_cur, n_par, 0, b.elems, kSplitTile, p->tile_meta);
     ++p->stats.launches;
-    if (!(l == 0 && fuse_hist)) {
+    if (!(l == 0 && fuse_hist) && !hist_ready) {
       GM_CUDA(cudaMemsetAsync(p->counts, 0, static_cast<size_t>(n_child) * sizeof(u32), st));
       k5_level<V, false><<<grid, kSplitThreads, split_smem_bytes<V>(false), st>>>(
-          xc, xv, b.elems, off_cur, n_par, p->tile_meta, F, prm.shift[l], p->counts, nullptr, nullptr, nullptr);
+          xc, xv, b.elems, off_cur, n_par, p->tile_meta, F, prm.shift[l], p->counts, nullptr, nullptr, nullptr, 0, 0, nullptr);
       ++p->stats.launches;
       GM_CUDA(cudaGetLastError());
     }
@@ -768,9 +769,13 @@ static int heavy_batch_front(gm_plan* p, const Batch& b, HeavyBatchState<V>* hs,
     p->stats.launches += 3;
     tm.end(st);
     tm.begin(PhaseTimes::kSplit, st);
+    // the counts of this level have been scanned: the array is free to receive the next level's
+    const bool next = l + 1 < prm.n_levels && !p->opts.separate_histogram;
+    if (next) GM_CUDA(cudaMemsetAsync(p->counts, 0, static_cast<size_t>(n_child) * prm.fanout[l + 1] * sizeof(u32), st));
     k5_level<V, true><<<grid, kSplitThreads, split_smem_bytes<V>(true), st>>>(
         xc, xv, b.elems, off_cur, n_par, p->tile_meta, F, prm.shift[l], nullptr, p->cursor, p->stage_col[cur ^ 1],
-        static_cast<V*>(p->stage_val[cur ^ 1]));
+        static_cast<V*>(p->stage_val[cur ^ 1]), next ? prm.fanout[l + 1] : 0, next ? prm.shift[l + 1] : 0, p->counts);
+    hist_ready = next;
     ++p->stats.launches;
     GM_CUDA(cudaGetLastError());
     tm.end(st);

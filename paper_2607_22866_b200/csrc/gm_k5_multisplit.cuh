@@ -17,6 +17,9 @@
 //                  child receives a contiguous, coalesced run.
 // A tile whose bins do not fit the shared table (very many tiny parents) falls back to one global
 // atomic per element.
+// When another level follows, the multisplit kernel also counts that level's (parent, child) bins while it writes
+// its tile out — the column is in a register and the element's child, which is the next level's parent, is known
+// — so deeper levels need no histogram pass over the staging buffer (4 bytes per product and a launch saved).
 #pragma once
 #include "gm_common.cuh"
 
@@ -33,9 +36,9 @@ constexpr int kSplitParentCap = kSplitThreads / 2;        // parents per tile on
 
 template <typename V>
 constexpr size_t split_smem_bytes(bool multisplit) {
-  // bins + parent offsets + parent starts (+ permuted columns and values)
+  // bins + parent offsets + parent starts (+ permuted columns and values + the next level's bins)
   size_t b = kSplitBinCap * 4 + (kSplitParentCap + 1) * 4 + kSplitParentCap * 4 + 64;
-  if (multisplit) b += static_cast<size_t>(kSplitTile) * (4 + sizeof(V));
+  if (multisplit) b += static_cast<size_t>(kSplitTile) * (4 + sizeof(V)) + kSplitBinCap * 4;
   return b;
 }
 
@@ -50,7 +53,9 @@ __global__ void __launch_bounds__(kSplitThreads, 1024 / kSplitThreads) k5_level(
     const i64* __restrict__ parent_off, i64 n_parents, const TileMeta* __restrict__ tile_meta, int F, int shift,
     u32* __restrict__ counts,     // histogram: (n_parents * F) counters, zero-initialised
     u64* __restrict__ cursor,     // multisplit: (n_parents * F) write cursors, start = child_off
-    int32_t* __restrict__ y_col, V* __restrict__ y_val) {
+    int32_t* __restrict__ y_col, V* __restrict__ y_val,
+    int next_F, int next_shift,   // multisplit: fan-out and shift of the level after this one (next_F == 0: none)
+    u32* __restrict__ next_counts) {  // ... and its (n_parents * F * next_F) counters, zero-initialised
   extern __shared__ __align__(16) unsigned char smem_raw[];
   u32* s_bin = reinterpret_cast<u32*>(smem_raw);                     // kSplitBinCap: counts -> starts -> deltas
   int* s_poff = reinterpret_cast<int*>(s_bin + kSplitBinCap);        // kSplitParentCap + 1: parent starts rel. to tile
@@ -58,6 +63,7 @@ __global__ void __launch_bounds__(kSplitThreads, 1024 / kSplitThreads) k5_level(
   V* s_val = reinterpret_cast<V*>(s_pstart + kSplitParentCap + 15);  // aligned below
   s_val = reinterpret_cast<V*>((reinterpret_cast<uintptr_t>(s_val)) & ~uintptr_t{15});
   int32_t* s_col = reinterpret_cast<int32_t*>(s_val + kSplitTile);
+  u32* s_next = reinterpret_cast<u32*>(s_col + kSplitTile);  // kSplitBinCap: (bin, next child) counts of the tile
   __shared__ u32 s_scan[33];
 
   const i64 t0 = static_cast<i64>(blockIdx.x) * kSplitTile;
@@ -89,6 +95,8 @@ __global__ void __launch_bounds__(kSplitThreads, 1024 / kSplitThreads) k5_level(
         const u64 dst = atomicAdd(&cursor[gbin], 1ull);
         y_col[dst] = c;
         y_val[dst] = x_val[p];
+        if (next_F > 0)
+          atomicAdd(&next_counts[gbin * next_F + ((static_cast<u32>(c) >> next_shift) & static_cast<u32>(next_F - 1))], 1u);
       } else {
         atomicAdd(&counts[gbin], 1u);
       }
@@ -233,33 +241,77 @@ __global__ void __launch_bounds__(kSplitThreads, 1024 / kSplitThreads) k5_level(
   }
   __syncthreads();
 
-  // ---- coalesced write: slot s belongs to the bin recomputed from its column and its parent
+  // ---- coalesced write: slot s belongs to the bin recomputed from its column and its parent.  The next level's
+  // bins are counted on the way: in shared memory when the tile's (bin, next child) pairs fit, else one global
+  // atomic per element.  Equal pairs sit next to each other (a bin's slots are contiguous and columns come in
+  // ascending runs), so the first lane of a run of equal pairs adds the run's length.
+  const bool count_next = MULTISPLIT && next_F > 0;
+  const bool next_in_smem = count_next && n_bins * next_F <= kSplitBinCap;
+  const u32 nmask = static_cast<u32>(next_F - 1);
+  if (next_in_smem) {
+    for (int b = tid; b < n_bins * next_F; b += kSplitThreads) s_next[b] = 0;
+    __syncthreads();
+  }
+  auto count_pair = [&](bool valid, u32 bin, int32_t c) {
+    if (!count_next) return;
+    const u32 pair = valid ? bin * static_cast<u32>(next_F) + ((static_cast<u32>(c) >> next_shift) & nmask) : 0xffffffffu;
+    const u32 prev = __shfl_up_sync(0xffffffffu, pair, 1);
+    const bool head = lane == 0 || pair != prev;
+    const u32 heads = __ballot_sync(0xffffffffu, head);
+    if (head && valid) {
+      const u32 above = heads & ~((2u << lane) - 1u);
+      const u32 len = static_cast<u32>((above ? __ffs(above) - 1 : 32) - static_cast<int>(lane));
+      if (next_in_smem) atomicAdd(&s_next[pair], len);
+      else atomicAdd(&next_counts[gbin0 * next_F + pair], len);
+    }
+  };
   if (n_par == 1) {
     // the usual tile (one parent): the bin is the child, nothing to search
-#pragma unroll 4
-    for (int s = tid; s < tn; s += kSplitThreads) {
-      const int32_t c = s_col[s];
-      const u32 dst = static_cast<u32>(s) + s_bin[(static_cast<u32>(c) >> shift) & fmask];
-      y_col[dst] = c;
-      y_val[dst] = s_val[s];
-    }
-    return;
-  }
-  for (int s = tid; s < tn; s += kSplitThreads) {
-    const int32_t c = s_col[s];
-    int par = 0;
-    {
-      int lo = 0, hi = n_par - 1;
-      while (lo < hi) {
-        const int mid = lo + ((hi - lo + 1) >> 1);
-        if (s_pstart[mid] <= s) lo = mid; else hi = mid - 1;
+    for (int s0 = 0; s0 < tn; s0 += kSplitThreads) {  // (whole warps stay in the loop: count_pair shuffles)
+      const int s = s0 + tid;
+      const bool valid = s < tn;
+      int32_t c = 0;
+      u32 bin = 0;
+      if (valid) {
+        c = s_col[s];
+        bin = (static_cast<u32>(c) >> shift) & fmask;
+        const u32 dst = static_cast<u32>(s) + s_bin[bin];
+        y_col[dst] = c;
+        y_val[dst] = s_val[s];
       }
-      par = lo;
+      count_pair(valid, bin, c);
     }
-    const u32 bin = static_cast<u32>(par * F) + ((static_cast<u32>(c) >> shift) & fmask);
-    const u32 dst = static_cast<u32>(s) + s_bin[bin];
-    y_col[dst] = c;
-    y_val[dst] = s_val[s];
+  } else {
+    for (int s0 = 0; s0 < tn; s0 += kSplitThreads) {
+      const int s = s0 + tid;
+      const bool valid = s < tn;
+      int32_t c = 0;
+      u32 bin = 0;
+      if (valid) {
+        c = s_col[s];
+        int par = 0;
+        {
+          int lo = 0, hi = n_par - 1;
+          while (lo < hi) {
+            const int mid = lo + ((hi - lo + 1) >> 1);
+            if (s_pstart[mid] <= s) lo = mid; else hi = mid - 1;
+          }
+          par = lo;
+        }
+        bin = static_cast<u32>(par * F) + ((static_cast<u32>(c) >> shift) & fmask);
+        const u32 dst = static_cast<u32>(s) + s_bin[bin];
+        y_col[dst] = c;
+        y_val[dst] = s_val[s];
+      }
+      count_pair(valid, bin, c);
+    }
+  }
+  if (next_in_smem) {
+    __syncthreads();
+    for (int b = tid; b < n_bins * next_F; b += kSplitThreads) {
+      const u32 cnt2 = s_next[b];
+      if (cnt2) atomicAdd(&next_counts[gbin0 * next_F + b], cnt2);
+    }
   }
 }
 

@@ -111,7 +111,11 @@ __global__ void k6_chunk_bases(const i64* __restrict__ chunk_nnz_off, i64 n_chun
 #define GM_SMALL_PER_LANE 16
 #endif
 constexpr int kSmallMaxPerLane = GM_SMALL_PER_LANE;
-constexpr int kAccSmallChunk = 32 * kSmallMaxPerLane;
+constexpr int kAccSmallChunk = 32 * kSmallMaxPerLane;  // largest chunk the one-warp sort can take
+// Default hand-over to the mid-size kernel.  The sort costs n log^2 n; measured on B200 (R-MAT scale 20 fp32 / scale 21
+// fp64, small + mid kernels together): 55 / 105 ms with chunks up to 512 products sorted, 50 / 90 ms up to 256,
+// 53 / 99 ms up to 128.
+constexpr int kAccSmallDefault = 256;
 constexpr int kSmallIdxBits = kSmallMaxPerLane == 32 ? 10 : (kSmallMaxPerLane == 16 ? 9 : 8);  // position of a product inside its chunk
 constexpr int kSmallWarps = 4;            // warps per block of the small-chunk kernel
 

@@ -42,31 +42,36 @@ __global__ void __launch_bounds__(kGatherThreads) k7_gather(
       }
     }
     __syncthreads();
-    // each thread walks kGatherTile / kGatherThreads positions strided by the block; its chunk index only grows.
-    // Positions are taken kGatherBatch at a time, all loads before the first store, so that a thread has that
-    // many independent loads in flight (one at a time left the kernel waiting on memory at full occupancy).
-    int cur = 0;
-    for (int q0 = threadIdx.x; q0 < tn; q0 += kGatherBatch * kGatherThreads) {
+    // A warp takes rows of 32 consecutive positions (row w, w + 8, ...), kGatherBatch rows at a time with all loads
+    // before the first store.  Chunks hold hundreds of entries on average, so a row usually lies inside one chunk:
+    // the warp keeps a uniform chunk cursor, and only a row that crosses a chunk boundary lets its lanes step on
+    // from there (the per-position binary search this replaces cost more instructions than the copy itself).
+    constexpr int kWarps = kGatherThreads / 32;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    int cur = 0;  // warp-uniform: last chunk whose start is <= the row's first position
+    for (int r0 = warp * 32; r0 < tn; r0 += kGatherBatch * kWarps * 32) {
       i64 dst[kGatherBatch];
       int32_t col[kGatherBatch];
       V val[kGatherBatch];
 #pragma unroll
       for (int u = 0; u < kGatherBatch; ++u) {
-        const int q = q0 + u * kGatherThreads;
+        const int q0 = r0 + u * kWarps * 32;
+        const int q = q0 + lane;
         dst[u] = -1;
-        if (q < tn) {
-          // last chunk whose start is <= q (empty chunks share a start with their successor and are skipped)
-          int lo = cur, hi = n_k - 1;
-          while (lo < hi) {
-            const int mid = lo + ((hi - lo + 1) >> 1);
-            if (s_rel[mid] <= q) lo = mid; else hi = mid - 1;
+        if (q0 < tn) {  // (uniform)
+          while (s_rel[cur + 1] <= q0) ++cur;  // empty chunks share a start with their successor and are skipped
+          int k = cur;
+          if (s_rel[cur + 1] < q0 + 32) {      // the row crosses into later chunks
+            if (q < tn)
+              while (s_rel[k + 1] <= q) ++k;
           }
-          cur = lo;
-          const i64 r = static_cast<i64>(q) - s_rel[cur];
-          dst[u] = s_dst[cur] + r;
-          const i64 src = s_src[cur] + r;
-          col[u] = s_col_in[src];
-          val[u] = s_val_in[src];
+          if (q < tn) {
+            const i64 r = static_cast<i64>(q) - s_rel[k];
+            dst[u] = s_dst[k] + r;
+            const i64 src = s_src[k] + r;
+            col[u] = s_col_in[src];
+            val[u] = s_val_in[src];
+          }
         }
       }
 #pragma unroll
