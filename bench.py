@@ -39,12 +39,14 @@ DEFAULT_CONFIG = 2  # R-MAT scale 20, edge factor 16, fp32: the largest fp32 pow
 
 
 # DRAM bytes per launch (ncu dram__bytes_read.sum + dram__bytes_write.sum) over the algorithmic bytes of the same
-# launch, from single-kernel, single-launch ncu captures of these kernels on the same product scaled down by 2**2
-# (R-MAT scale 18, one batch of 0.5-0.8 G products, about 4 GB on the device).  Traffic grows in proportion to the
-# products processed, so a full-size launch is its algorithmic figure times this ratio.  A kernel that has changed
-# since its capture has no entry (traffic is then reported as null).
-TRAFFIC_RATIO = {}
-TRAFFIC_SOURCE = "single-launch ncu captures on R-MAT scale 18 (same recipe, 2**2 smaller), scaled by products"
+# launch, from single-kernel, single-launch ncu captures of these kernels on the same product scaled down by 2**3
+# (R-MAT scale 17: one batch holds the whole product, 1.09 G products, about 9 GB staged).  Traffic grows in
+# proportion to the products processed, so a full-size launch is its algorithmic figure times this ratio.  A kernel
+# that has changed since its capture must lose its entry (traffic is then reported as null).
+TRAFFIC_RATIO = {"k4_expand": 1.04, "k5a_histogram": 1.00, "k5b_multisplit": 1.00, "k6_small_chunks": 0.66,
+                 "k6_mid_chunks": 0.99, "k6_accumulate": 1.00, "k7_gather": 1.00}
+TRAFFIC_SOURCE = ("single-kernel, single-launch ncu DRAM-counter captures on the same recipe 2**3 smaller (R-MAT scale 17, "
+                  "one batch holds the whole product), scaled by products")
 
 
 def ctypes_copy(dst, src):
