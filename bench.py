@@ -53,6 +53,25 @@ def ctypes_copy(dst, src):
     ctypes.memmove(ctypes.byref(dst), ctypes.byref(src), ctypes.sizeof(src))
 
 
+def max_over_ranks(ms_local: float, world: int, device) -> float:
+    """Step time of a multi-rank run: every rank times its own replica on its device, the job's time is the slowest
+    rank's (MAX all-reduce; the backend is whatever the process group was made with)."""
+    if world <= 1:
+        return float(ms_local)
+    import torch
+    import torch.distributed as dist
+
+    t = torch.tensor([ms_local], device=device, dtype=torch.float64)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def replicas_value(products_per_replica: int, world: int, ms_step: float) -> float:
+    """Whole-job GFLOP/s of `world` independent replicas ("replicas only": no data-path collective): all ranks'
+    products over the slowest rank's time."""
+    return world * 2.0 * products_per_replica / (ms_step * 1e-3) / 1e9
+
+
 def _peaks():
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(path):
@@ -355,10 +374,7 @@ def main():
         ev1.record()
         barrier()
         clocks = sampler.stop() if sampler else None
-        t = torch.tensor([ev0.elapsed_time(ev1)], device="cuda", dtype=torch.float64)
-        if world > 1:
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms_step = float(t.item()) / steps
+        ms_step = max_over_ranks(ev0.elapsed_time(ev1), world, "cuda") / steps
         products = int(info.products_total)
         stats_avg = {k: v / steps for k, v in stats_sum.items()}
         # byte model: the row analysis (untimed plan) says which entries of A sit in light rows
@@ -368,7 +384,7 @@ def main():
         n_light_entries_a = int(np.diff(A.row_ptr)[ip_dev <= info.params.tau].sum())
         kt = kernel_table(info, stats_avg, sv, B.nnz, n_light_entries_a)
         dom = max(kt, key=lambda k: kt[k]["ms"])
-        return {"ms_step": ms_step, "value": world * 2.0 * products / (ms_step * 1e-3) / 1e9, "products": products,
+        return {"ms_step": ms_step, "value": replicas_value(products, world, ms_step), "products": products,
                 "info": info, "kernels": kt, "dominant": dom, "launches": launches, "nnz": int(nnz), "clocks": clocks}
 
     peak, peak_kind = _peaks()

@@ -42,6 +42,9 @@ def compare_rows(C, ref, dtype, r0=0):
 
 
 def check_product(A, B, smem_bytes=232448, **opts):
+    # debug mode on unless the test says otherwise: inputs validated on the device, and every product checked to lie in
+    # the columns its chunk owns before it is accumulated (a misplaced product would otherwise be folded in silently)
+    opts.setdefault("validate_inputs", 1)
     C, info, stats = run_gpu(A, B, smem_bytes, **opts)
     ref = oracle.spgemm(A, B)
     assert C.n_rows == A.n_rows and C.n_cols == B.n_cols

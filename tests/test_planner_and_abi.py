@@ -169,3 +169,31 @@ def test_bench_reference_arm_under_torchrun_two_ranks():
     rec = json.loads(lines[0])
     assert rec["impl"] == "reference" and rec["n_gpus"] == 2 and rec["cpu_baseline"]["kind"] == "oracle"
     assert rec["value"] > 0 and rec["e2e"]["h2d_bytes_per_step"] == 0
+
+
+def _gloo_rank(rank, world, port, out):
+    import torch.distributed as dist
+    os.environ["MASTER_ADDR"], os.environ["MASTER_PORT"] = "127.0.0.1", str(port)
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    sys.path.insert(0, ROOT)
+    import bench
+    ms = bench.max_over_ranks(100.0 + 50.0 * rank, world, "cpu")     # rank 1 is the slow replica
+    dist.barrier()
+    out.put((rank, ms, bench.replicas_value(10 ** 9, world, ms)))
+    dist.destroy_process_group()
+
+
+def test_replica_timing_takes_the_slowest_rank_gloo_two_ranks():
+    # "replicas only": the job's step time is the maximum over ranks and the aggregate counts every rank's products
+    import torch.multiprocessing as mp
+    ctx = mp.get_context("spawn")
+    out = ctx.Queue()
+    procs = [ctx.Process(target=_gloo_rank, args=(r, 2, 29733, out)) for r in range(2)]
+    for p in procs:
+        p.start()
+    got = sorted(out.get(timeout=120) for _ in procs)
+    for p in procs:
+        p.join(timeout=60)
+        assert p.exitcode == 0
+    assert [g[1] for g in got] == [150.0, 150.0]
+    assert abs(got[0][2] - 2 * 2.0 * 1e9 / 0.150 / 1e9) < 1e-9 and got[0][2] == got[1][2]
