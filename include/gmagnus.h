@@ -97,7 +97,11 @@ typedef struct gm_plan_opts {
                               the call returns GM_ERR_TIMEOUT (0 = the default, about four million).  Negative:
                               the copies are announced but withheld, so the wait runs out after that many polls
                               with nothing in flight (how the tests reach the time-out path)                     */
-  int32_t reserved[2];
+  int32_t expand_order;    /* 1: the expansion runs in outer-product order (Eq. 2, Algorithm 4 as printed): the
+                              batch's segments are sorted by row of B (masked CSR->CSC), so a row of B is read once
+                              for all heavy rows that use it; the first multisplit level then runs as separate
+                              passes.  0 (default): row order                                                   */
+  int32_t reserved[1];
 } gm_plan_opts;
 
 /* What the host planner derives from (C.m, value size, smem_bytes): Section III-D. */

@@ -45,7 +45,7 @@ class PlanOpts(ctypes.Structure):
                 ("validate_inputs", ctypes.c_int32), ("single_stream", ctypes.c_int32),
                 ("level0_multisplit", ctypes.c_int32), ("small_chunk_max", ctypes.c_int32),
                 ("mid_chunk_max", ctypes.c_int32), ("expand_staging", ctypes.c_int32),
-                ("debug_spin_limit", ctypes.c_int32), ("reserved", ctypes.c_int32 * 2)]
+                ("debug_spin_limit", ctypes.c_int32), ("expand_order", ctypes.c_int32), ("reserved", ctypes.c_int32 * 1)]
 
 
 class Params(ctypes.Structure):

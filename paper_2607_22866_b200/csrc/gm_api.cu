@@ -15,6 +15,7 @@
 #include "gm_k4_expand.cuh"
 #include "gm_k4_direct.cuh"
 #include "gm_k4_stream.cuh"
+#include "gm_k4_csc.cuh"
 #include "gm_k5_multisplit.cuh"
 #include "gm_k6_accumulate.cuh"
 #include "gm_k7_gather.cuh"
@@ -169,6 +170,14 @@ struct gm_plan {
   bool stream = false;             // ... with the rows of B brought in by bulk copies (needs 16-byte aligned B arrays)
   int32_t* seg_hrow = nullptr;     // n_seg: heavy row (position in the heavy-row list) of every segment
   uint32_t* seg_rec = nullptr;     // segment records of a batch for the bulk-copy expansion (run starts + entry of A)
+  // outer-product (CSC) order of the expansion, option expand_order = 1: per batch, the segments sorted by row of B
+  bool csc = false;
+  int32_t* csc_cnt = nullptr;      // n_rows(B) + 1: segments per row of B
+  int64_t* csc_ptr = nullptr;      // n_rows(B) + 1: their exclusive scan (the masked CSC's column pointer)
+  gm::u64* csc_cursor = nullptr;   // n_rows(B) + 1: scatter cursors
+  int32_t* csc_perm = nullptr;     // segments of a batch in CSC order
+  int32_t* csc_len = nullptr;      // their product counts
+  int64_t* csc_off = nullptr;      // ... and the exclusive scan: the flattened product space in CSC order
   int small_max = 0, mid_max = 0;  // size classes of the final chunks: <= small_max one warp, <= mid_max one small block
   std::vector<int64_t> heavy_nz_off_host;
   int64_t* heavy_nz_off = nullptr; // nH + 1
@@ -403,7 +412,8 @@ static int build_plan(gm_plan* p, cudaStream_t st) {
     // buffer of the default size takes)
     const i64 bound_bytes = prm.n_levels > 0 ? B.n_rows * static_cast<i64>(prm.fanout[0] + 1) * 4 : 0;
     const bool bounds_fit = bound_bytes <= std::max<i64>(i64{1} << 30, std::min<i64>(info.products_heavy, i64{1} << 29) * (4 + p->sv));
-    p->direct = prm.n_levels > 0 && prm.fanout[0] <= 256 &&
+    p->csc = p->opts.expand_order == 1;
+    p->direct = prm.n_levels > 0 && prm.fanout[0] <= 256 && !p->csc &&
                 (p->opts.level0_multisplit == 2 || (p->opts.level0_multisplit == 0 && long_segments && bounds_fit));
     info.level0_direct = p->direct ? 1 : 0;
     {
@@ -478,8 +488,21 @@ static int build_plan(gm_plan* p, cudaStream_t st) {
         ++info.launches;
       }
     }
+    i64 csc_scan_len = 0;
+    if (p->csc) {
+      i64 max_seg_b = 0;
+      for (const Batch& b : p->batches)
+        max_seg_b = std::max(max_seg_b, p->heavy_nz_off_host[static_cast<size_t>(b.h1)] - p->heavy_nz_off_host[static_cast<size_t>(b.h0)]);
+      GM_TRY(plan_alloc(p, &p->csc_cnt, static_cast<size_t>(B.n_rows) + 1, st));
+      GM_TRY(plan_alloc(p, &p->csc_ptr, static_cast<size_t>(B.n_rows) + 2, st));
+      GM_TRY(plan_alloc(p, &p->csc_cursor, static_cast<size_t>(B.n_rows) + 2, st));
+      GM_TRY(plan_alloc(p, &p->csc_perm, static_cast<size_t>(max_seg_b) + 1, st));
+      GM_TRY(plan_alloc(p, &p->csc_len, static_cast<size_t>(max_seg_b) + 1, st));
+      GM_TRY(plan_alloc(p, &p->csc_off, static_cast<size_t>(max_seg_b) + 2, st));
+      csc_scan_len = std::max<i64>(B.n_rows, max_seg_b);
+    }
     int64_t* tmp2 = nullptr;  // the per-batch scans can be longer than the ones above
-    GM_TRY(plan_alloc(p, &tmp2, static_cast<size_t>(scan_tmp_elems(std::max<i64>({static_cast<i64>(n_chunks_max), nnzA, nA, 1}))), st));
+    GM_TRY(plan_alloc(p, &tmp2, static_cast<size_t>(scan_tmp_elems(std::max<i64>({static_cast<i64>(n_chunks_max), nnzA, nA, csc_scan_len, 1}))), st));
     p->scan_tmp = tmp2;
   }
   GM_CUDA(cudaStreamSynchronize(st));
@@ -718,8 +741,30 @@ static int heavy_batch_front(gm_plan* p, const Batch& b, HeavyBatchState<V>* hs,
     first_level = 1;
   }
   // the expansion kernel counts the first level's (row, child) bins while it writes, unless asked not to
-  const bool fuse_hist = !p->direct && prm.n_levels > 0 && !p->opts.separate_histogram;
-  if (!p->direct) {
+  const bool fuse_hist = !p->direct && prm.n_levels > 0 && !p->opts.separate_histogram && !p->csc;
+  if (p->csc) {
+    // ---- outer-product order: masked CSR -> CSC of the batch's segments (counting sort by row of B), then the
+    // expansion walks the product space in that order
+    tm.begin(PhaseTimes::kExpand, st);
+    const i64 seg0 = p->heavy_nz_off_host[static_cast<size_t>(b.h0)];
+    const i64 n_seg_b = p->heavy_nz_off_host[static_cast<size_t>(b.h1)] - seg0;
+    const i64 nB = p->B.n_rows;
+    GM_CUDA(cudaMemsetAsync(p->csc_cnt, 0, static_cast<size_t>(nB + 1) * sizeof(int32_t), st));
+    k_csc_count<<<grid_for(n_seg_b, 256, p->num_sms, 16), 256, 0, st>>>(p->seg_brow, seg0, n_seg_b, p->csc_cnt);
+    exclusive_scan<int32_t, i64>(p->csc_cnt, p->csc_ptr, nB, p->scan_tmp, nullptr, nullptr, reinterpret_cast<i64*>(p->csc_cursor), st);
+    k_csc_scatter<<<grid_for(n_seg_b, 256, p->num_sms, 16), 256, 0, st>>>(p->seg_brow, p->seg_off, seg0, n_seg_b, p->csc_cursor,
+                                                                          p->csc_perm, p->csc_len);
+    exclusive_scan<int32_t, i64>(p->csc_len, p->csc_off, n_seg_b, p->scan_tmp, nullptr, nullptr, nullptr, st);
+    const unsigned grid = static_cast<unsigned>((b.elems + kExpandTile - 1) / kExpandTile);
+    k_tile_bounds<<<grid_for(grid, 256, p->num_sms), 256, 0, st>>>(p->csc_off, n_seg_b, 0, b.elems, kExpandTile, p->tile_meta);
+    k4_expand_csc<V><<<grid, kExpandThreads, 0, st>>>(p->csc_off, p->csc_perm, p->seg_off, p->seg_bstart, p->seg_j, seg0,
+                                                      p->tile_meta, static_cast<const V*>(p->A.vals), p->B.col_idx,
+                                                      static_cast<const V*>(p->B.vals), b.elem0, b.elems, p->stage_col[0],
+                                                      static_cast<V*>(p->stage_val[0]));
+    p->stats.launches += 10;
+    GM_CUDA(cudaGetLastError());
+    tm.end(st);
+  } else if (!p->direct) {
   tm.begin(PhaseTimes::kExpand, st);
   {
     static_assert(kExpandTile == kSplitTile, "the fused histogram shares the multisplit's tiles");
@@ -743,7 +788,9 @@ static int heavy_batch_front(gm_plan* p, const Batch& b, HeavyBatchState<V>* hs,
   tm.end(st);
   }
   if (prm.n_levels > first_level) {
-    GM_CUDA(cudaFuncSetAttribute(k5_level<V, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+    GM_CUDA(cudaFuncSetAttribute(k5_level<V, true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 static_cast<int>(split_smem_bytes<V>(true))));
+    GM_CUDA(cudaFuncSetAttribute(k5_level<V, true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                  static_cast<int>(split_smem_bytes<V>(true))));
   }
   bool hist_ready = false;  // the previous level's multisplit counted this level's bins while it wrote
@@ -772,9 +819,15 @@ static int heavy_batch_front(gm_plan* p, const Batch& b, HeavyBatchState<V>* hs,
     // the counts of this level have been scanned: the array is free to receive the next level's
     const bool next = l + 1 < prm.n_levels && !p->opts.separate_histogram;
     if (next) GM_CUDA(cudaMemsetAsync(p->counts, 0, static_cast<size_t>(n_child) * prm.fanout[l + 1] * sizeof(u32), st));
-    k5_level<V, true><<<grid, kSplitThreads, split_smem_bytes<V>(true), st>>>(
-        xc, xv, b.elems, off_cur, n_par, p->tile_meta, F, prm.shift[l], nullptr, p->cursor, p->stage_col[cur ^ 1],
-        static_cast<V*>(p->stage_val[cur ^ 1]), next ? prm.fanout[l + 1] : 0, next ? prm.shift[l + 1] : 0, p->counts);
+    if (next) {
+      k5_level<V, true, true><<<grid, kSplitThreads, split_smem_bytes<V>(true), st>>>(
+          xc, xv, b.elems, off_cur, n_par, p->tile_meta, F, prm.shift[l], nullptr, p->cursor, p->stage_col[cur ^ 1],
+          static_cast<V*>(p->stage_val[cur ^ 1]), prm.fanout[l + 1], prm.shift[l + 1], p->counts);
+    } else {
+      k5_level<V, true, false><<<grid, kSplitThreads, split_smem_bytes<V>(true), st>>>(
+          xc, xv, b.elems, off_cur, n_par, p->tile_meta, F, prm.shift[l], nullptr, p->cursor, p->stage_col[cur ^ 1],
+          static_cast<V*>(p->stage_val[cur ^ 1]), 0, 0, nullptr);
+    }
     hist_ready = next;
     ++p->stats.launches;
     GM_CUDA(cudaGetLastError());

@@ -47,7 +47,7 @@ struct SplitTileInfo {
   int n_par;  // parents touching the tile (including empty ones in between)
 };
 
-template <typename V, bool MULTISPLIT>
+template <typename V, bool MULTISPLIT, bool NEXT = false>  // NEXT: the multisplit also counts the next level's bins
 __global__ void __launch_bounds__(kSplitThreads, 1024 / kSplitThreads) k5_level(
     const int32_t* __restrict__ x_col, const V* __restrict__ x_val, i64 n_elems,
     const i64* __restrict__ parent_off, i64 n_parents, const TileMeta* __restrict__ tile_meta, int F, int shift,
@@ -95,7 +95,7 @@ __global__ void __launch_bounds__(kSplitThreads, 1024 / kSplitThreads) k5_level(
         const u64 dst = atomicAdd(&cursor[gbin], 1ull);
         y_col[dst] = c;
         y_val[dst] = x_val[p];
-        if (next_F > 0)
+        if (NEXT)
           atomicAdd(&next_counts[gbin * next_F + ((static_cast<u32>(c) >> next_shift) & static_cast<u32>(next_F - 1))], 1u);
       } else {
         atomicAdd(&counts[gbin], 1u);
@@ -245,7 +245,7 @@ __global__ void __launch_bounds__(kSplitThreads, 1024 / kSplitThreads) k5_level(
   // bins are counted on the way: in shared memory when the tile's (bin, next child) pairs fit, else one global
   // atomic per element.  Equal pairs sit next to each other (a bin's slots are contiguous and columns come in
   // ascending runs), so the first lane of a run of equal pairs adds the run's length.
-  const bool count_next = MULTISPLIT && next_F > 0;
+  constexpr bool count_next = MULTISPLIT && NEXT;
   const bool next_in_smem = count_next && n_bins * next_F <= kSplitBinCap;
   const u32 nmask = static_cast<u32>(next_F - 1);
   if (next_in_smem) {
@@ -253,7 +253,7 @@ __global__ void __launch_bounds__(kSplitThreads, 1024 / kSplitThreads) k5_level(
     __syncthreads();
   }
   auto count_pair = [&](bool valid, u32 bin, int32_t c) {
-    if (!count_next) return;
+    if constexpr (!count_next) return;
     const u32 pair = valid ? bin * static_cast<u32>(next_F) + ((static_cast<u32>(c) >> next_shift) & nmask) : 0xffffffffu;
     const u32 prev = __shfl_up_sync(0xffffffffu, pair, 1);
     const bool head = lane == 0 || pair != prev;
@@ -265,6 +265,36 @@ __global__ void __launch_bounds__(kSplitThreads, 1024 / kSplitThreads) k5_level(
       else atomicAdd(&next_counts[gbin0 * next_F + pair], len);
     }
   };
+  if constexpr (!count_next) {
+    if (n_par == 1) {
+      // the usual tile (one parent): the bin is the child, nothing to search
+#pragma unroll 4
+      for (int s = tid; s < tn; s += kSplitThreads) {
+        const int32_t c = s_col[s];
+        const u32 dst = static_cast<u32>(s) + s_bin[(static_cast<u32>(c) >> shift) & fmask];
+        y_col[dst] = c;
+        y_val[dst] = s_val[s];
+      }
+      return;
+    }
+    for (int s = tid; s < tn; s += kSplitThreads) {
+      const int32_t c = s_col[s];
+      int par = 0;
+      {
+        int lo = 0, hi = n_par - 1;
+        while (lo < hi) {
+          const int mid = lo + ((hi - lo + 1) >> 1);
+          if (s_pstart[mid] <= s) lo = mid; else hi = mid - 1;
+        }
+        par = lo;
+      }
+      const u32 bin = static_cast<u32>(par * F) + ((static_cast<u32>(c) >> shift) & fmask);
+      const u32 dst = static_cast<u32>(s) + s_bin[bin];
+      y_col[dst] = c;
+      y_val[dst] = s_val[s];
+    }
+    return;
+  }
   if (n_par == 1) {
     // the usual tile (one parent): the bin is the child, nothing to search
     for (int s0 = 0; s0 < tn; s0 += kSplitThreads) {  // (whole warps stay in the loop: count_pair shuffles)

@@ -404,6 +404,25 @@ def test_bounded_wait_on_bulk_copies_runs_out_cleanly():
     check_product(A, A, expand_staging=1, **kw)
 
 
+@pytest.mark.parametrize("dtype,width,fanout", [(np.float32, 8192, 0), (np.float64, 512, 16), (np.float32, 128, 8)])
+def test_outer_product_order_expansion(dtype, width, fanout):
+    # expand_order = 1: the batch's segments sorted by row of B (masked CSR -> CSC), products generated column of A by
+    # column of A as in Eq. 2 / Algorithm 4; zero, one and two multisplit levels, several batches
+    A = gen.rmat(13, 16, seed=17, dtype=dtype)
+    kw = dict(tau=256, chunk_width=width, stage_elems=1 << 20)
+    if fanout:
+        kw["max_fanout"] = fanout
+    C1, info, _ = check_product(A, A, expand_order=1, **kw)
+    assert info.level0_direct == 0 and info.n_batches > 1
+    C2, _, _ = run_gpu(A, A, **kw)
+    assert torch.equal(C1.row_ptr, C2.row_ptr) and torch.equal(C1.col, C2.col)
+    # rows of B of 0 to 3 entries: tiles with more segments than the shared window holds, empty segments
+    rng = np.random.default_rng(29)
+    Bs = random_csr(rng, 3000, 5000, 0.0004, dtype)
+    As = random_csr(rng, 40, 3000, 0.6, dtype)
+    check_product(As, Bs, tau=64, chunk_width=256, max_fanout=4, expand_order=1)
+
+
 def test_expansion_straight_into_the_first_level_short_rows_of_b():
     # rows of B with 0 to 3 entries: tiles with thousands of segments, empty segments, heavy rows made of them
     rng = np.random.default_rng(23)
