@@ -238,7 +238,11 @@ def kernel_table(info, stats_avg, sv, nnz_b, n_light_entries_a):
     # that level, only per-segment run starts (read two child-boundary rows of B, write one row of prefixes)
     l0 = 1 if (L > 0 and info.level0_direct) else 0
     hist = sum(4 * e + 8 * (parents[l] + 1) + 4 * parents[l + 1] for l in range(l0, L))
-    split = sum(2 * se * e + 8 * (parents[l] + 1) + 8 * parents[l + 1] for l in range(l0, L))
+    # a multisplit pass reads every column of the batch and moves (reads the value of, writes) only the products of
+    # chunks that have not left the hierarchy early
+    moved = stats_avg["split_products"]
+    split = (2 * se * moved + 4 * ((L - l0) * e - moved)
+             + sum(8 * (parents[l] + 1) + 8 * parents[l + 1] for l in range(l0, L)))
     seg_tables = (12 * p.fanout[0] * info.nnz_a_heavy + 4 * parents[1]) if l0 else 0
     tbl = {
         "k3_light_symbolic": (4 * n_light_entries_a + 8 * info.rows_light + 4 * nnz_b, stats_avg["ms_light_symbolic"]),
@@ -385,7 +389,8 @@ def main():
         kt = kernel_table(info, stats_avg, sv, B.nnz, n_light_entries_a)
         dom = max(kt, key=lambda k: kt[k]["ms"])
         return {"ms_step": ms_step, "value": replicas_value(products, world, ms_step), "products": products,
-                "info": info, "kernels": kt, "dominant": dom, "launches": launches, "nnz": int(nnz), "clocks": clocks}
+                "info": info, "kernels": kt, "dominant": dom, "launches": launches, "nnz": int(nnz), "clocks": clocks,
+                "early_exit_products": int(stats_avg["early_exit_products"])}
 
     peak, peak_kind = _peaks()
     m = measure(A, B, dA, dB, opts, args.steps, args.warmup, True)
@@ -415,7 +420,8 @@ def main():
                    "products": products, "products_heavy": int(info.products_heavy), "nnz_c": int(nnz),
                    "rows_heavy": int(info.rows_heavy), "tau": int(tau), "chunk_width": int(info.params.chunk_width),
                    "levels": info.params.levels(), "batches": int(info.n_batches), "smem_bytes": SMEM_BYTES,
-                   "level0_direct": int(info.level0_direct), "plan_opts": args.opt,
+                   "level0_direct": int(info.level0_direct),
+                   "early_exit_products": m["early_exit_products"], "plan_opts": args.opt,
                    "step": "gm_spgemm_plan + gm_spgemm_execute (C freed after each step)"},
         "roofline": roofline, "kernels": kt, "clocks": clocks, "gpu_launches": launches,
     }

@@ -101,7 +101,11 @@ typedef struct gm_plan_opts {
                               batch's segments are sorted by row of B (masked CSR->CSC), so a row of B is read once
                               for all heavy rows that use it; the first multisplit level then runs as separate
                               passes.  0 (default): row order                                                   */
-  int32_t reserved[1];
+  int32_t early_exit;      /* Algorithm 3's early exit (only heavy chunks recurse): from the second level on, a chunk
+                              with at most this many products is not split further; it stays in the level's input
+                              buffer and is accumulated by the one-warp sort over its whole column span.  0 =
+                              default (small_chunk_max), -1 = every chunk goes through every level, at most
+                              small_chunk_max                                                                  */
 } gm_plan_opts;
 
 /* What the host planner derives from (C.m, value size, smem_bytes): Section III-D. */
@@ -154,6 +158,9 @@ typedef struct gm_exec_stats {
   float reserved[3];
   int64_t mid_chunk_products;  /* products in chunks handled by the one-small-block-per-chunk kernel             */
   int64_t mid_chunk_entries;   /* entries of C those chunks produced                                             */
+  int64_t early_exit_products; /* products of chunks that left the multisplit hierarchy before its last level    */
+  int64_t early_exit_chunks;   /* ... and how many chunks did                                                     */
+  int64_t split_products;      /* products moved by multisplit passes, summed over the levels                     */
 } gm_exec_stats;
 
 typedef struct gm_plan gm_plan; /* opaque, owned by the library */

@@ -45,7 +45,7 @@ class PlanOpts(ctypes.Structure):
                 ("validate_inputs", ctypes.c_int32), ("single_stream", ctypes.c_int32),
                 ("level0_multisplit", ctypes.c_int32), ("small_chunk_max", ctypes.c_int32),
                 ("mid_chunk_max", ctypes.c_int32), ("expand_staging", ctypes.c_int32),
-                ("debug_spin_limit", ctypes.c_int32), ("expand_order", ctypes.c_int32), ("reserved", ctypes.c_int32 * 1)]
+                ("debug_spin_limit", ctypes.c_int32), ("expand_order", ctypes.c_int32), ("early_exit", ctypes.c_int32)]
 
 
 class Params(ctypes.Structure):
@@ -76,7 +76,9 @@ class ExecStats(ctypes.Structure):
                 ("ms_expand", ctypes.c_float), ("ms_histogram", ctypes.c_float), ("ms_multisplit", ctypes.c_float),
                 ("ms_accumulate", ctypes.c_float), ("ms_gather", ctypes.c_float), ("ms_scan", ctypes.c_float),
                 ("ms_total", ctypes.c_float), ("ms_small_chunks", ctypes.c_float), ("ms_mid_chunks", ctypes.c_float),
-                ("reserved", ctypes.c_float * 3), ("mid_chunk_products", ctypes.c_int64), ("mid_chunk_entries", ctypes.c_int64)]
+                ("reserved", ctypes.c_float * 3), ("mid_chunk_products", ctypes.c_int64), ("mid_chunk_entries", ctypes.c_int64),
+                ("early_exit_products", ctypes.c_int64), ("early_exit_chunks", ctypes.c_int64),
+                ("split_products", ctypes.c_int64)]
 
 
 _ALLOC_FN = ctypes.CFUNCTYPE(ctypes.c_void_p, ctypes.c_size_t, ctypes.c_void_p, ctypes.c_void_p)

@@ -179,6 +179,9 @@ struct gm_plan {
   int32_t* csc_len = nullptr;      // their product counts
   int64_t* csc_off = nullptr;      // ... and the exclusive scan: the flattened product space in CSC order
   int small_max = 0, mid_max = 0;  // size classes of the final chunks: <= small_max one warp, <= mid_max one small block
+  int exit_max = -1;               // chunks of at most this many products leave the multisplit hierarchy early (-1: none)
+  unsigned char* exit_tag[2]{};    // per (parent, child) of a level: where the chunk left the hierarchy (ping-pong)
+  unsigned char* parent_tag = nullptr;  // per parent of the level that runs: != 0, not split
   std::vector<int64_t> heavy_nz_off_host;
   int64_t* heavy_nz_off = nullptr; // nH + 1
   int32_t* sym_rows = nullptr;     // bins x nA
@@ -188,7 +191,8 @@ struct gm_plan {
   int32_t* row_nnz = nullptr;      // nA
   int64_t* scan_tmp = nullptr;
   int64_t* c_total = nullptr;      // [0] running nnz(C) (device carry), [1] heavy entries, [2] products and [3] entries of
-                                   // small chunks, [4] products and [5] entries of mid-size chunks
+                                   // small chunks, [4] products and [5] entries of mid-size chunks, [6] products and
+                                   // [7] chunks that left the hierarchy early, [8] products the levels did not move
   int* err = nullptr;
   // heavy workspace
   int32_t* stage_col[2]{};
@@ -290,6 +294,11 @@ static int build_plan(gm_plan* p, cudaStream_t st) {
     // several mid-chunk blocks must fit an SM next to each other for the class to pay
     while (mid > p->small_max && mid_smem_bytes(prm.chunk_width, p->sv, mid) + 1024 > p->smem_bytes / 8) mid /= 2;
     p->mid_max = std::max(mid, p->small_max);
+    if (o.early_exit < -1 || o.early_exit > kAccSmallChunk) return fail(GM_ERR_INVALID_ARG, "early_exit out of range");
+    // early exit needs the one-warp sort (the only accumulate kernel that takes a chunk wider than W) and a level
+    // after the first
+    p->exit_max = (o.early_exit < 0 || p->small_max <= 0 || prm.n_levels < 2) ? -1
+                  : std::min(o.early_exit ? o.early_exit : p->small_max, p->small_max);
   }
 
   GM_TRY(plan_alloc(p, &p->err, 4, st));
@@ -318,7 +327,7 @@ static int build_plan(gm_plan* p, cudaStream_t st) {
   GM_TRY(plan_alloc(p, &heavy_pos, static_cast<size_t>(nA) + 1, st));
   GM_TRY(plan_alloc(p, &totals, 1, st));
   GM_TRY(plan_alloc(p, &p->row_nnz, static_cast<size_t>(nA) + 1, st));
-  GM_TRY(plan_alloc(p, &p->c_total, 8, st));
+  GM_TRY(plan_alloc(p, &p->c_total, 16, st));
   GM_TRY(plan_alloc(p, &p->scan_tmp, static_cast<size_t>(scan_tmp_elems(std::max<i64>(std::max(nnzA, nA), 1))), st));
   GM_CUDA(cudaMemsetAsync(totals, 0, sizeof(K1Totals), st));
   if (nnzA > 0) k1_nz_len<<<grid_for(nnzA, 256, p->num_sms, 32), 256, 0, st>>>(A.col_idx, nnzA, B.row_ptr, nz_len);
@@ -468,6 +477,11 @@ static int build_plan(gm_plan* p, cudaStream_t st) {
     GM_TRY(plan_alloc(p, &p->mid_list, n_chunks_max + 1, st));
     GM_TRY(plan_alloc(p, &p->big_list, n_chunks_max + 1, st));
     GM_TRY(plan_alloc(p, &p->acc_counters, 8, st));
+    if (p->exit_max >= 0) {
+      GM_TRY(plan_alloc(p, &p->exit_tag[0], n_chunks_max + 1, st));
+      GM_TRY(plan_alloc(p, &p->exit_tag[1], n_chunks_max + 1, st));
+      GM_TRY(plan_alloc(p, &p->parent_tag, n_chunks_max + 1, st));
+    }
     const size_t n_tiles_max = static_cast<size_t>(info.stage_elems) / std::min({kExpandTile, kSplitTile, kGatherTile}) + 2;
     GM_TRY(plan_alloc(p, &p->tile_meta, n_tiles_max, st));
     GM_TRY(plan_alloc(p, &p->row_meta, n_tiles_max, st));
@@ -578,6 +592,11 @@ struct HeavyBatchState {
   const i64* chunk_off = nullptr;    // n_chunks + 1 batch-relative offsets
   i64 n_chunks = 0;
   int log2_cpr = 0;
+  // chunks that left the multisplit hierarchy early (tags == nullptr: none can have)
+  const unsigned char* tags = nullptr;
+  int32_t* alt_col = nullptr;  // the staging buffer that is not fin_col
+  V* alt_val = nullptr;
+  ExitTags xt;
 };
 
 // K6: accumulate every chunk of the batch and compact it in place; chunk_nnz receives the entry counts.
@@ -591,8 +610,8 @@ static int launch_accumulate(gm_plan* p, const Batch& b, const HeavyBatchState<V
   GM_CUDA(cudaMemsetAsync(p->acc_counters, 0, 8 * sizeof(int), st));
   GM_CUDA(cudaMemsetAsync(p->chunk_nnz, 0, static_cast<size_t>(hs.n_chunks) * sizeof(u32), st));
   if (p->opts.validate_inputs) {
-    k6_validate_chunks<<<grid_for(hs.n_chunks * 32, 256, p->num_sms, 8), 256, 0, st>>>(hs.fin_col, hs.chunk_off, hs.n_chunks,
-                                                                                      hs.log2_cpr, W, p->B.n_cols, p->err);
+    k6_validate_chunks<<<grid_for(hs.n_chunks * 32, 256, p->num_sms, 8), 256, 0, st>>>(
+        hs.fin_col, hs.chunk_off, hs.n_chunks, hs.log2_cpr, W, p->B.n_cols, p->err, hs.tags, hs.alt_col, hs.xt);
     ++p->stats.launches;
   }
   k6_classify<<<grid_for(hs.n_chunks, 256, p->num_sms), 256, 0, st>>>(hs.chunk_off, hs.n_chunks, small_max, mid_max, p->mid_list,
@@ -602,7 +621,7 @@ static int launch_accumulate(gm_plan* p, const Batch& b, const HeavyBatchState<V
     p->times.begin(PhaseTimes::kAccSmall, st);
     k6_small_chunks<V><<<static_cast<unsigned>(p->num_sms * 8), kSmallWarps * 32, 0, st>>>(
         hs.fin_col, hs.fin_val, hs.chunk_off, hs.n_chunks, W, small_max, p->chunk_nnz,
-        reinterpret_cast<u64*>(p->c_total + 2));
+        reinterpret_cast<u64*>(p->c_total + 2), hs.tags, hs.alt_col, hs.alt_val, hs.xt);
     ++p->stats.launches;
     p->times.end(st);
   }
@@ -653,8 +672,13 @@ static int launch_gather(gm_plan* p, const Batch& b, const HeavyBatchState<V>& h
   const unsigned grid = static_cast<unsigned>((b.elems + kGatherTile - 1) / kGatherTile);
   k_tile_bounds<<<grid_for(grid, 256, p->num_sms), 256, 0, st>>>(p->chunk_nnz_off, hs.n_chunks, 0, 0, kGatherTile,
                                                                p->tile_meta, p->chunk_nnz_off + hs.n_chunks);
-  k7_gather<V><<<grid, kGatherThreads, 0, st>>>(hs.fin_col, hs.fin_val, hs.chunk_off, p->chunk_nnz_off, p->chunk_base,
-                                                hs.n_chunks, p->tile_meta, c_col, c_val, c_capacity, p->err);
+  if (hs.tags && hs.xt.alt_bits)
+    k7_gather<V, true><<<grid, kGatherThreads, 0, st>>>(hs.fin_col, hs.fin_val, hs.chunk_off, p->chunk_nnz_off, p->chunk_base,
+                                                        hs.n_chunks, p->tile_meta, c_col, c_val, c_capacity, p->err,
+                                                        hs.alt_col, hs.alt_val, hs.tags, hs.xt.alt_bits);
+  else
+    k7_gather<V><<<grid, kGatherThreads, 0, st>>>(hs.fin_col, hs.fin_val, hs.chunk_off, p->chunk_nnz_off, p->chunk_base,
+                                                  hs.n_chunks, p->tile_meta, c_col, c_val, c_capacity, p->err);
   p->stats.launches += 3;
   GM_CUDA(cudaGetLastError());
   return GM_OK;
@@ -792,8 +816,16 @@ static int heavy_batch_front(gm_plan* p, const Batch& b, HeavyBatchState<V>* hs,
                                  static_cast<int>(split_smem_bytes<V>(true))));
     GM_CUDA(cudaFuncSetAttribute(k5_level<V, true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                  static_cast<int>(split_smem_bytes<V>(true))));
+    GM_CUDA(cudaFuncSetAttribute(k5_level<V, true, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 static_cast<int>(split_smem_bytes<V>(true))));
+    GM_CUDA(cudaFuncSetAttribute(k5_level<V, true, true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 static_cast<int>(split_smem_bytes<V>(true))));
   }
   bool hist_ready = false;  // the previous level's multisplit counted this level's bins while it wrote
+  // early exit: tags of the current parents (none before the first level that can leave chunks behind)
+  const unsigned char* tag_cur = nullptr;
+  int tag_buf = 0;
+  int level_buf[GM_MAX_LEVELS + 1] = {0};  // staging buffer a level read from
   for (int l = first_level; l < prm.n_levels; ++l) {
     const int F = prm.fanout[l];
     const i64 n_child = n_par * F;
@@ -810,6 +842,22 @@ static int heavy_batch_front(gm_plan* p, const Batch& b, HeavyBatchState<V>* hs,
       ++p->stats.launches;
       GM_CUDA(cudaGetLastError());
     }
+    // Early exit: a parent of a level after the first that holds few products stays where it is; its span of columns
+    // must still fit the sort's packed key
+    level_buf[l] = cur;
+    const int span_bits = prm.shift[l] + ilog2_floor(static_cast<uint64_t>(F));
+    const bool can_exit = p->exit_max >= 0 && l >= 1 && span_bits + kSmallIdxBits <= 32;
+    const bool exiting = can_exit || tag_cur != nullptr;
+    if (exiting) {
+      unsigned char* tag_nxt = p->exit_tag[tag_buf];
+      k5_exit_flags<<<grid_for(n_child, 256, p->num_sms, 32), 256, 0, st>>>(
+          off_cur, n_par, ilog2_floor(static_cast<uint64_t>(F)), tag_cur, can_exit ? p->exit_max : -1, l + 1, p->counts,
+          p->parent_tag, tag_nxt, reinterpret_cast<u64*>(p->c_total + 6));
+      ++p->stats.launches;
+      tag_cur = tag_nxt;
+      tag_buf ^= 1;
+      hs->xt.set(l + 1, false, span_bits);  // (which buffer: known once the last level has run)
+    }
     tm.end(st);
     tm.begin(PhaseTimes::kScan, st);
     exclusive_scan<u32, i64>(p->counts, off_nxt, n_child, p->scan_tmp, nullptr, nullptr, reinterpret_cast<i64*>(p->cursor), st);
@@ -819,7 +867,15 @@ static int heavy_batch_front(gm_plan* p, const Batch& b, HeavyBatchState<V>* hs,
     // the counts of this level have been scanned: the array is free to receive the next level's
     const bool next = l + 1 < prm.n_levels && !p->opts.separate_histogram;
     if (next) GM_CUDA(cudaMemsetAsync(p->counts, 0, static_cast<size_t>(n_child) * prm.fanout[l + 1] * sizeof(u32), st));
-    if (next) {
+    if (exiting && next) {
+      k5_level<V, true, true, true><<<grid, kSplitThreads, split_smem_bytes<V>(true), st>>>(
+          xc, xv, b.elems, off_cur, n_par, p->tile_meta, F, prm.shift[l], nullptr, p->cursor, p->stage_col[cur ^ 1],
+          static_cast<V*>(p->stage_val[cur ^ 1]), prm.fanout[l + 1], prm.shift[l + 1], p->counts, p->parent_tag);
+    } else if (exiting) {
+      k5_level<V, true, false, true><<<grid, kSplitThreads, split_smem_bytes<V>(true), st>>>(
+          xc, xv, b.elems, off_cur, n_par, p->tile_meta, F, prm.shift[l], nullptr, p->cursor, p->stage_col[cur ^ 1],
+          static_cast<V*>(p->stage_val[cur ^ 1]), 0, 0, nullptr, p->parent_tag);
+    } else if (next) {
       k5_level<V, true, true><<<grid, kSplitThreads, split_smem_bytes<V>(true), st>>>(
           xc, xv, b.elems, off_cur, n_par, p->tile_meta, F, prm.shift[l], nullptr, p->cursor, p->stage_col[cur ^ 1],
           static_cast<V*>(p->stage_val[cur ^ 1]), prm.fanout[l + 1], prm.shift[l + 1], p->counts);
@@ -828,6 +884,7 @@ static int heavy_batch_front(gm_plan* p, const Batch& b, HeavyBatchState<V>* hs,
           xc, xv, b.elems, off_cur, n_par, p->tile_meta, F, prm.shift[l], nullptr, p->cursor, p->stage_col[cur ^ 1],
           static_cast<V*>(p->stage_val[cur ^ 1]), 0, 0, nullptr);
     }
+    p->stats.split_products += b.elems;
     hist_ready = next;
     ++p->stats.launches;
     GM_CUDA(cudaGetLastError());
@@ -841,6 +898,13 @@ static int heavy_batch_front(gm_plan* p, const Batch& b, HeavyBatchState<V>* hs,
   hs->chunk_off = off_cur;
   hs->n_chunks = n_par;
   hs->log2_cpr = ilog2_floor(static_cast<uint64_t>(prm.chunks_required));
+  hs->tags = tag_cur;
+  if (tag_cur) {
+    hs->alt_col = p->stage_col[cur ^ 1];
+    hs->alt_val = static_cast<V*>(p->stage_val[cur ^ 1]);
+    for (int l = 1; l < prm.n_levels; ++l)
+      if (level_buf[l] != cur) hs->xt.alt_bits |= 1u << (l + 1);
+  }
   p->stats.final_chunks += n_par;
   p->stats.staged_products += b.elems;
 
@@ -879,7 +943,7 @@ static int execute_t(gm_plan* p, cudaStream_t st, gm_csr* C) {
 
   GM_CUDA(cudaMemsetAsync(p->err, 0, sizeof(int), st));
   GM_CUDA(cudaMemsetAsync(p->row_nnz, 0, static_cast<size_t>(nA + 1) * sizeof(int32_t), st));
-  GM_CUDA(cudaMemsetAsync(p->c_total, 0, 8 * sizeof(int64_t), st));
+  GM_CUDA(cudaMemsetAsync(p->c_total, 0, 16 * sizeof(int64_t), st));
 
   // ---- result row_ptr
   i64* c_row_ptr = static_cast<i64*>(dev_alloc(static_cast<size_t>(nA + 1) * sizeof(i64), st));
@@ -1062,8 +1126,10 @@ static int execute_t(gm_plan* p, cudaStream_t st, gm_csr* C) {
     }
   }
   if (tm.enabled) cudaEventRecord(ev_total1, st);
-  i64 tail_totals[5] = {0, 0, 0, 0, 0};  // heavy entries; products and entries of small chunks; of mid-size chunks
-  cudaMemcpyAsync(tail_totals, p->c_total + 1, 5 * sizeof(i64), cudaMemcpyDeviceToHost, st);
+  // heavy entries; products and entries of small chunks; of mid-size chunks; products and chunks that left the
+  // hierarchy early; products the multisplit levels left in place
+  i64 tail_totals[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+  cudaMemcpyAsync(tail_totals, p->c_total + 1, 8 * sizeof(i64), cudaMemcpyDeviceToHost, st);
   cudaError_t e1 = cudaMemcpyAsync(&dev_err, p->err, sizeof(int), cudaMemcpyDeviceToHost, st);
   cudaError_t e2 = cudaStreamSynchronize(st);
   if (e1 != cudaSuccess || e2 != cudaSuccess) {
@@ -1083,6 +1149,9 @@ static int execute_t(gm_plan* p, cudaStream_t st, gm_csr* C) {
   p->stats.small_chunk_entries = tail_totals[2];
   p->stats.mid_chunk_products = tail_totals[3];
   p->stats.mid_chunk_entries = tail_totals[4];
+  p->stats.early_exit_products = tail_totals[5];
+  p->stats.early_exit_chunks = tail_totals[6];
+  p->stats.split_products -= tail_totals[7];
   p->stats.c_capacity = capacity;
   if (tm.enabled) {
     float ph[PhaseTimes::kCount];

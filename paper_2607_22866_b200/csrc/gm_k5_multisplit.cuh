@@ -20,6 +20,15 @@
 // When another level follows, the multisplit kernel also counts that level's (parent, child) bins while it writes
 // its tile out — the column is in a register and the element's child, which is the next level's parent, is known
 // — so deeper levels need no histogram pass over the staging buffer (4 bytes per product and a launch saved).
+//
+// Early exit (Algorithm 3: only heavy chunks recurse; Section III-A: light chunks take their own accumulation
+// branch).  From the second level on, a parent that holds few products is not split any further: its products stay
+// where they are, in the level's *input* buffer, and the parent's whole range is booked to its child 0 all the way
+// down, so the chunk table keeps its regular (row, chunk) shape and the parent's range in either staging buffer
+// stays its own.  k5_exit_flags marks such parents and rewrites their row of the count matrix; the multisplit
+// kernel (EXIT) drops their products before ranking, loads no values for them and returns at once from a tile
+// that holds nothing else.  The final chunks carry the tag of the level they left at, from which the accumulate and
+// gather kernels know the buffer and the column span.
 #pragma once
 #include "gm_common.cuh"
 
@@ -38,7 +47,7 @@ template <typename V>
 constexpr size_t split_smem_bytes(bool multisplit) {
   // bins + parent offsets + parent starts (+ permuted columns and values + the next level's bins)
   size_t b = kSplitBinCap * 4 + (kSplitParentCap + 1) * 4 + kSplitParentCap * 4 + 64;
-  if (multisplit) b += static_cast<size_t>(kSplitTile) * (4 + sizeof(V)) + kSplitBinCap * 4;
+  if (multisplit) b += static_cast<size_t>(kSplitTile) * (4 + sizeof(V)) + kSplitBinCap * 4 + kSplitParentCap;
   return b;
 }
 
@@ -47,7 +56,46 @@ struct SplitTileInfo {
   int n_par;  // parents touching the tile (including empty ones in between)
 };
 
-template <typename V, bool MULTISPLIT, bool NEXT = false>  // NEXT: the multisplit also counts the next level's bins
+// Marks the parents of a level that leave the hierarchy here (tag != 0) and books their products to child 0.
+// One thread per (parent, child).  tag_in: the parents' tags from the level before (NULL at the first level that
+// can exit); a parent that left earlier keeps its tag.  counts: the level's count matrix, already filled.
+__global__ void k5_exit_flags(const i64* __restrict__ parent_off, i64 n_parents, int log2F,
+                              const unsigned char* __restrict__ tag_in, int exit_max, int level_tag,
+                              u32* __restrict__ counts, unsigned char* __restrict__ parent_tag,
+                              unsigned char* __restrict__ child_tag,
+                              u64* __restrict__ totals) {  // [0] += products, [1] += parents that leave at this level,
+                                                           // [2] += products that this level does not move
+  const i64 n_child = n_parents << log2F;
+  u64 prod = 0, par = 0, stay = 0;
+  for (i64 i = static_cast<i64>(blockIdx.x) * blockDim.x + threadIdx.x; i < n_child;
+       i += static_cast<i64>(gridDim.x) * blockDim.x) {
+    const i64 P = i >> log2F;
+    const int c = static_cast<int>(i & ((i64{1} << log2F) - 1));
+    const i64 n = parent_off[P + 1] - parent_off[P];
+    int tag = tag_in ? tag_in[P] : 0;
+    if (!tag && n <= exit_max) {
+      tag = level_tag;
+      if (c == 0 && n > 0) { prod += static_cast<u64>(n); ++par; }
+    }
+    if (tag && c == 0) stay += static_cast<u64>(n);
+    child_tag[i] = static_cast<unsigned char>(tag);
+    if (c == 0) parent_tag[P] = static_cast<unsigned char>(tag);
+    if (tag) counts[i] = c == 0 ? static_cast<u32>(n) : 0u;
+  }
+  for (int o = 16; o > 0; o >>= 1) {
+    prod += __shfl_xor_sync(0xffffffffu, prod, o);
+    par += __shfl_xor_sync(0xffffffffu, par, o);
+    stay += __shfl_xor_sync(0xffffffffu, stay, o);
+  }
+  if ((threadIdx.x & 31) == 0 && stay) {
+    if (prod) atomicAdd(&totals[0], prod);
+    if (par) atomicAdd(&totals[1], par);
+    atomicAdd(&totals[2], stay);
+  }
+}
+
+// NEXT: the multisplit also counts the next level's bins.  EXIT: parents with parent_tag != 0 are left where they are.
+template <typename V, bool MULTISPLIT, bool NEXT = false, bool EXIT = false>
 __global__ void __launch_bounds__(kSplitThreads, 1024 / kSplitThreads) k5_level(
     const int32_t* __restrict__ x_col, const V* __restrict__ x_val, i64 n_elems,
     const i64* __restrict__ parent_off, i64 n_parents, const TileMeta* __restrict__ tile_meta, int F, int shift,
@@ -55,7 +103,8 @@ __global__ void __launch_bounds__(kSplitThreads, 1024 / kSplitThreads) k5_level(
     u64* __restrict__ cursor,     // multisplit: (n_parents * F) write cursors, start = child_off
     int32_t* __restrict__ y_col, V* __restrict__ y_val,
     int next_F, int next_shift,   // multisplit: fan-out and shift of the level after this one (next_F == 0: none)
-    u32* __restrict__ next_counts) {  // ... and its (n_parents * F * next_F) counters, zero-initialised
+    u32* __restrict__ next_counts,    // ... and its (n_parents * F * next_F) counters, zero-initialised
+    const unsigned char* __restrict__ parent_tag = nullptr) {  // EXIT: per parent, != 0: not split at this level
   extern __shared__ __align__(16) unsigned char smem_raw[];
   u32* s_bin = reinterpret_cast<u32*>(smem_raw);                     // kSplitBinCap: counts -> starts -> deltas
   int* s_poff = reinterpret_cast<int*>(s_bin + kSplitBinCap);        // kSplitParentCap + 1: parent starts rel. to tile
@@ -64,6 +113,7 @@ __global__ void __launch_bounds__(kSplitThreads, 1024 / kSplitThreads) k5_level(
   s_val = reinterpret_cast<V*>((reinterpret_cast<uintptr_t>(s_val)) & ~uintptr_t{15});
   int32_t* s_col = reinterpret_cast<int32_t*>(s_val + kSplitTile);
   u32* s_next = reinterpret_cast<u32*>(s_col + kSplitTile);  // kSplitBinCap: (bin, next child) counts of the tile
+  unsigned char* s_ptag = reinterpret_cast<unsigned char*>(s_next + kSplitBinCap);  // kSplitParentCap: tags of the tile's parents
   __shared__ u32 s_scan[33];
 
   const i64 t0 = static_cast<i64>(blockIdx.x) * kSplitTile;
@@ -84,11 +134,20 @@ __global__ void __launch_bounds__(kSplitThreads, 1024 / kSplitThreads) k5_level(
   const i64 p_lo = tm.first;
   const u32 fmask = static_cast<u32>(F - 1);
 
+  if constexpr (EXIT && MULTISPLIT) {
+    // a tile of many small parents that all stay behind (the usual tile once a level's chunks are light) moves nothing
+    if (tm.n > 2) {
+      int moves = 0;
+      for (int k = tid; k < tm.n; k += kSplitThreads) moves |= parent_tag[p_lo + k] == 0;
+      if (!__syncthreads_or(moves)) return;
+    }
+  }
   if (tm.n > kSplitParentCap || static_cast<i64>(tm.n) * F > kSplitBinCap) {
     // ---- slow path: one global atomic per element
     for (int q = tid; q < tn; q += kSplitThreads) {
       const i64 p = t0 + q;
       const i64 par = last_le(parent_off, p_lo, p_lo + tm.n - 1, p);
+      if (EXIT && MULTISPLIT && parent_tag[par]) continue;
       const int32_t c = x_col[p];  // (the hoisted registers are striped differently; this path is rare)
       const i64 gbin = par * F + ((static_cast<u32>(c) >> shift) & fmask);
       if (MULTISPLIT) {
@@ -111,6 +170,14 @@ __global__ void __launch_bounds__(kSplitThreads, 1024 / kSplitThreads) k5_level(
   if (n_par > 2)
     for (int k = tid; k <= n_par; k += kSplitThreads)
       s_poff[k] = (k == n_par) ? tn + 1 : clamp_rel(parent_off[p_lo + k] - t0, -1, tn + 1);
+  bool ex0 = false, ex1 = false;  // EXIT: the tile's first two parents stay behind
+  if constexpr (EXIT && MULTISPLIT) {
+    ex0 = parent_tag[p_lo] != 0;
+    ex1 = n_par > 1 ? parent_tag[p_lo + 1] != 0 : true;
+    if (n_par <= 2 && ex0 && ex1) return;  // (uniform) nothing of this tile moves
+    if (n_par > 2)
+      for (int k = tid; k < n_par; k += kSplitThreads) s_ptag[k] = parent_tag[p_lo + k];
+  }
   __syncthreads();
 
   // ---- local histogram; every element learns its rank inside its bin
@@ -131,6 +198,10 @@ __global__ void __launch_bounds__(kSplitThreads, 1024 / kSplitThreads) k5_level(
         par = lo;
       }
       bin = static_cast<u32>(par * F) + ((static_cast<u32>(col[k]) >> shift) & fmask);
+      if constexpr (EXIT && MULTISPLIT) {
+        const bool stay = n_par > 2 ? s_ptag[par] != 0 : (par ? ex1 : ex0);
+        if (stay) bin = 0xffffffffu;
+      }
     }
     // Rank inside the bin.  A shared-memory atomic that returns its old value costs one wavefront per lane
     // that hits the same address, and with few bins (or one hot child) that is every lane.  So the lanes of a
@@ -176,6 +247,7 @@ __global__ void __launch_bounds__(kSplitThreads, 1024 / kSplitThreads) k5_level(
       if (bin != 0xffffffffu) atomicAdd(&s_bin[bin], 1u);
     }
     rank_bin[k] = (rank << 11) | (bin & 2047u);
+    if (EXIT && bin == 0xffffffffu) rank_bin[k] = 0xffffffffu;  // (a rank never reaches 2^21 - 1: not a valid pair)
   }
   __syncthreads();
 
@@ -200,6 +272,7 @@ __global__ void __launch_bounds__(kSplitThreads, 1024 / kSplitThreads) k5_level(
   }
   u32 total;
   u32 start = block_exclusive_scan(sum, s_scan, &total);
+  const int tv = EXIT ? static_cast<int>(total) : tn;  // elements of the tile that move
   u32 delta[kBinsPerThread];
 #pragma unroll
   for (int k = 0; k < kBinsPerThread; ++k) {
@@ -220,12 +293,12 @@ __global__ void __launch_bounds__(kSplitThreads, 1024 / kSplitThreads) k5_level(
 #pragma unroll
     for (int k = 0; k < 8; ++k) {
       const int q = (h + k) * kSplitThreads + tid;
-      if (q < tn) v[k] = x_val[t0 + q];
+      if (q < tn && !(EXIT && rank_bin[h + k] == 0xffffffffu)) v[k] = x_val[t0 + q];
     }
 #pragma unroll
     for (int k = 0; k < 8; ++k) {
       const int q = (h + k) * kSplitThreads + tid;
-      if (q < tn) {
+      if (q < tn && !(EXIT && rank_bin[h + k] == 0xffffffffu)) {
         const u32 rb = rank_bin[h + k];
         const u32 dst = s_bin[rb & 2047u] + (rb >> 11);
         s_col[dst] = col[h + k];
@@ -269,7 +342,7 @@ __global__ void __launch_bounds__(kSplitThreads, 1024 / kSplitThreads) k5_level(
     if (n_par == 1) {
       // the usual tile (one parent): the bin is the child, nothing to search
 #pragma unroll 4
-      for (int s = tid; s < tn; s += kSplitThreads) {
+      for (int s = tid; s < tv; s += kSplitThreads) {
         const int32_t c = s_col[s];
         const u32 dst = static_cast<u32>(s) + s_bin[(static_cast<u32>(c) >> shift) & fmask];
         y_col[dst] = c;
@@ -277,7 +350,7 @@ __global__ void __launch_bounds__(kSplitThreads, 1024 / kSplitThreads) k5_level(
       }
       return;
     }
-    for (int s = tid; s < tn; s += kSplitThreads) {
+    for (int s = tid; s < tv; s += kSplitThreads) {
       const int32_t c = s_col[s];
       int par = 0;
       {
@@ -297,9 +370,9 @@ __global__ void __launch_bounds__(kSplitThreads, 1024 / kSplitThreads) k5_level(
   }
   if (n_par == 1) {
     // the usual tile (one parent): the bin is the child, nothing to search
-    for (int s0 = 0; s0 < tn; s0 += kSplitThreads) {  // (whole warps stay in the loop: count_pair shuffles)
+    for (int s0 = 0; s0 < tv; s0 += kSplitThreads) {  // (whole warps stay in the loop: count_pair shuffles)
       const int s = s0 + tid;
-      const bool valid = s < tn;
+      const bool valid = s < tv;
       int32_t c = 0;
       u32 bin = 0;
       if (valid) {
@@ -312,9 +385,9 @@ __global__ void __launch_bounds__(kSplitThreads, 1024 / kSplitThreads) k5_level(
       count_pair(valid, bin, c);
     }
   } else {
-    for (int s0 = 0; s0 < tn; s0 += kSplitThreads) {
+    for (int s0 = 0; s0 < tv; s0 += kSplitThreads) {
       const int s = s0 + tid;
-      const bool valid = s < tn;
+      const bool valid = s < tv;
       int32_t c = 0;
       u32 bin = 0;
       if (valid) {

@@ -30,6 +30,20 @@
 
 namespace gm {
 
+// Where the chunks that left the multisplit hierarchy early live.  A final chunk's tag (0: it went through every
+// level) is 1 + the level whose pass left it behind; per tag, one bit says whether that level's input was the
+// other staging buffer than the one the last level wrote, and five bits give log2 of the columns the chunk spans.
+struct ExitTags {
+  u32 alt_bits = 0;
+  u64 span_pack = 0;
+  __host__ __device__ bool alt(int tag) const { return (alt_bits >> tag) & 1u; }
+  __host__ __device__ int span_bits(int tag) const { return static_cast<int>((span_pack >> (5 * tag)) & 31u); }
+  void set(int tag, bool other_buffer, int bits) {
+    if (other_buffer) alt_bits |= 1u << tag;
+    span_pack |= static_cast<u64>(bits) << (5 * tag);
+  }
+};
+
 constexpr int kMidThreads = 128;        // threads of one mid-chunk team
 constexpr int kHugeChunk = 1 << 16;     // big chunks with more products than this are handed out first
 
@@ -70,18 +84,25 @@ __global__ void k6_classify(const i64* __restrict__ chunk_off, i64 n_chunks, int
 // Debug net (plan option validate_inputs): every product that reaches the accumulate kernels must lie in the W
 // columns its chunk owns.  One warp per chunk; a violation sets kDevBadChunk (the kernels themselves mask the
 // column and would fold a misplaced product into the wrong entry silently).
+// Chunks that left the hierarchy early (tag != 0, see ExitTags) own the columns of all the final chunks they stand for.
 __global__ void k6_validate_chunks(const int32_t* __restrict__ x_col, const i64* __restrict__ chunk_off, i64 n_chunks,
-                                   int log2_chunks_per_row, int W, i64 n_cols, int* __restrict__ err) {
+                                   int log2_chunks_per_row, int W, i64 n_cols, int* __restrict__ err,
+                                   const unsigned char* __restrict__ tags, const int32_t* __restrict__ x_col_alt,
+                                   ExitTags xt) {
   const int lane = threadIdx.x & 31;
   const int log2W = 31 - __clz(W);
   const u32 crow_mask = (1u << log2_chunks_per_row) - 1u;
   const i64 n_warps = static_cast<i64>(gridDim.x) * (blockDim.x >> 5);
   for (i64 k = static_cast<i64>(blockIdx.x) * (blockDim.x >> 5) + (threadIdx.x >> 5); k < n_chunks; k += n_warps) {
-    const u32 want = static_cast<u32>(k) & crow_mask;
+    const int tag = tags ? tags[k] : 0;
+    const int32_t* col = tag && xt.alt(tag) ? x_col_alt : x_col;
+    const int bits = tag ? xt.span_bits(tag) : log2W;  // columns the chunk owns: 2^bits
+    const u32 want = (static_cast<u32>(k) & crow_mask) >> (bits - log2W);
     bool bad = false;
     for (i64 q = chunk_off[k] + lane; q < chunk_off[k + 1]; q += 32) {
-      const int32_t c = x_col[q];
-      bad |= c < 0 || c >= n_cols || (static_cast<u32>(c) >> log2W) != want;
+      const int32_t c = col[q];
+      bad |= c < 0 || c >= n_cols || (static_cast<u32>(c) >> bits) != want ||
+             (static_cast<u32>(k) & ((1u << (bits - log2W)) - 1u)) != 0;  // an early chunk's products sit in its first slot
     }
     if (bad) dev_set_error(err, kDevBadChunk);
   }
@@ -173,7 +194,7 @@ __device__ __forceinline__ void warp_sort_keys(u32 (&key)[K], int lane) {
 // One small chunk by one warp.  s_key / s_val: 32 * K entries of this warp's shared memory.
 template <typename V, int K>
 __device__ __forceinline__ int small_chunk(int32_t* col, V* val, int n, u32 wmask, u32* s_key, V* s_val,
-                                           u32* nnz_out) {
+                                           u32* nnz_out, int32_t c_row0, V v_row0) {  // (the caller loaded element `lane`)
   const int lane = threadIdx.x & 31;
   u32 key[K];
   int32_t c_first = 0;
@@ -182,10 +203,10 @@ __device__ __forceinline__ int small_chunk(int32_t* col, V* val, int n, u32 wmas
     const int e = r * 32 + lane;
     key[r] = 0xffffffffu;  // padding sorts to the end
     if (e < n) {
-      const int32_t c = col[e];
+      const int32_t c = r == 0 ? c_row0 : col[e];
       if (e == 0) c_first = c;
       key[r] = ((static_cast<u32>(c) & wmask) << kSmallIdxBits) | static_cast<u32>(e);
-      s_val[e] = val[e];
+      s_val[e] = r == 0 ? v_row0 : val[e];
     }
   }
   const u32 col_base = static_cast<u32>(__shfl_sync(0xffffffffu, c_first, 0)) & ~wmask;
@@ -222,10 +243,12 @@ __device__ __forceinline__ int small_chunk(int32_t* col, V* val, int n, u32 wmas
 }
 
 template <typename V>
-__global__ void __launch_bounds__(kSmallWarps * 32) k6_small_chunks(
+__global__ void __launch_bounds__(kSmallWarps * 32, 8) k6_small_chunks(
     int32_t* x_col, V* x_val, const i64* __restrict__ chunk_off, i64 n_chunks, int W, int small_max,
     u32* __restrict__ chunk_nnz,
-    u64* __restrict__ totals) {  // [0] += products, [1] += entries of the chunks handled here (statistics)
+    u64* __restrict__ totals,  // [0] += products, [1] += entries of the chunks handled here (statistics)
+    const unsigned char* __restrict__ tags,  // per chunk, or NULL: != 0 for chunks that left the hierarchy early
+    int32_t* x_col_alt, V* x_val_alt, ExitTags xt) {
   __shared__ u32 s_key[kSmallWarps][32 * kSmallMaxPerLane];
   __shared__ V s_val[kSmallWarps][32 * kSmallMaxPerLane];
   const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
@@ -237,28 +260,58 @@ __global__ void __launch_bounds__(kSmallWarps * 32) k6_small_chunks(
   for (i64 g = static_cast<i64>(blockIdx.x) * kSmallWarps + w; g < n_groups; g += static_cast<i64>(gridDim.x) * kSmallWarps) {
     const i64 k = (g << 5) + lane;
     i64 cs = 0;
-    int cn = 0;
+    int cn = 0, ctag = 0;
     if (k < n_chunks) {
       cs = chunk_off[k];
       cn = static_cast<int>(min(chunk_off[k + 1] - cs, static_cast<i64>(INT_MAX)));
+      if (tags) ctag = tags[k];
     }
     u32 todo = __ballot_sync(0xffffffffu, cn > 0 && cn <= small_max);
-    while (todo) {
-      const int src = __ffs(todo) - 1;
-      todo &= todo - 1;
+    if (!todo) continue;
+    // A chunk's work starts with a round trip to HBM and the warp has nothing else to do meanwhile, so the first 32
+    // products of the next chunk are requested before the current chunk is sorted (most small chunks hold no more).
+    struct Job {
+      int32_t* col;
+      V* val;
+      int n, src;
+      u32 wm;
+      int32_t c0;
+      V v0;
+    };
+    auto open_job = [&](int src) {
+      Job j;
       const i64 s0 = __shfl_sync(0xffffffffu, cs, src);
-      const int n = __shfl_sync(0xffffffffu, cn, src);
-      int32_t* col = x_col + s0;
-      V* val = x_val + s0;
-      u32* out = &chunk_nnz[(g << 5) + src];
+      j.n = __shfl_sync(0xffffffffu, cn, src);
+      j.src = src;
+      const int tag = __shfl_sync(0xffffffffu, ctag, src);
+      // an early chunk lies in the buffer it was left in and is sorted over all the columns it spans
+      const bool alt = tag && xt.alt(tag);
+      j.col = (alt ? x_col_alt : x_col) + s0;
+      j.val = (alt ? x_val_alt : x_val) + s0;
+      j.wm = tag ? (1u << xt.span_bits(tag)) - 1u : wmask;
+      j.c0 = 0;
+      j.v0 = V(0);
+      if (lane < j.n) { j.c0 = j.col[lane]; j.v0 = j.val[lane]; }
+      return j;
+    };
+    Job cur = open_job(__ffs(todo) - 1);
+    todo &= todo - 1;
+    for (;;) {
+      const bool more = todo != 0;  // (uniform)
+      Job nxt = cur;
+      if (more) { nxt = open_job(__ffs(todo) - 1); todo &= todo - 1; }
+      const int n = cur.n;
+      u32* out = &chunk_nnz[(g << 5) + cur.src];
       int m;
-      if (n <= 32) m = small_chunk<V, 1>(col, val, n, wmask, s_key[w], s_val[w], out);
-      else if (n <= 64) m = small_chunk<V, 2>(col, val, n, wmask, s_key[w], s_val[w], out);
-      else if (n <= 128) m = small_chunk<V, 4>(col, val, n, wmask, s_key[w], s_val[w], out);
-      else if (kSmallMaxPerLane == 8 || n <= 256) m = small_chunk<V, 8>(col, val, n, wmask, s_key[w], s_val[w], out);
-      else if (kSmallMaxPerLane == 16 || n <= 512) m = small_chunk<V, (kSmallMaxPerLane >= 16 ? 16 : 8)>(col, val, n, wmask, s_key[w], s_val[w], out);
-      else m = small_chunk<V, kSmallMaxPerLane>(col, val, n, wmask, s_key[w], s_val[w], out);
+      if (n <= 32) m = small_chunk<V, 1>(cur.col, cur.val, n, cur.wm, s_key[w], s_val[w], out, cur.c0, cur.v0);
+      else if (n <= 64) m = small_chunk<V, 2>(cur.col, cur.val, n, cur.wm, s_key[w], s_val[w], out, cur.c0, cur.v0);
+      else if (n <= 128) m = small_chunk<V, 4>(cur.col, cur.val, n, cur.wm, s_key[w], s_val[w], out, cur.c0, cur.v0);
+      else if (kSmallMaxPerLane == 8 || n <= 256) m = small_chunk<V, 8>(cur.col, cur.val, n, cur.wm, s_key[w], s_val[w], out, cur.c0, cur.v0);
+      else if (kSmallMaxPerLane == 16 || n <= 512) m = small_chunk<V, (kSmallMaxPerLane >= 16 ? 16 : 8)>(cur.col, cur.val, n, cur.wm, s_key[w], s_val[w], out, cur.c0, cur.v0);
+      else m = small_chunk<V, kSmallMaxPerLane>(cur.col, cur.val, n, cur.wm, s_key[w], s_val[w], out, cur.c0, cur.v0);
       if (lane == 0) { s_sum[w][0] += static_cast<u64>(n); s_sum[w][1] += static_cast<u64>(m); }
+      if (!more) break;
+      cur = nxt;
     }
   }
   if (lane == 0 && s_sum[w][0]) {

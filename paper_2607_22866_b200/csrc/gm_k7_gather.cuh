@@ -4,6 +4,8 @@
 // batch (prefix sums of chunk_nnz) is cut into equal tiles, one per block; a thread finds the chunk
 // of its output position in a shared-memory copy of the tile's chunk table, so both the reads and
 // the writes are contiguous runs.  Pure streaming: 2 * (4 + value bytes) per entry.
+// ALT: chunks that left the multisplit hierarchy early may lie in the other staging buffer (see ExitTags); their
+// table entry carries a flag bit and the copy reads from there.
 #pragma once
 #include "gm_common.cuh"
 
@@ -19,12 +21,16 @@ constexpr int kGatherTile = 4096;
 constexpr int kGatherBatch = GM_GATHER_BATCH;
 constexpr int kGatherChunkCap = 1024;  // chunks staged in shared memory per tile; more -> per-element search
 
-template <typename V>
+constexpr i64 kGatherAltBit = i64{1} << 62;
+
+template <typename V, bool ALT = false>
 __global__ void __launch_bounds__(kGatherThreads) k7_gather(
     const int32_t* __restrict__ s_col_in, const V* __restrict__ s_val_in,  // staging buffer (compacted chunks)
     const i64* __restrict__ chunk_off, const i64* __restrict__ chunk_nnz_off, const i64* __restrict__ chunk_base,
     i64 n_chunks, const TileMeta* __restrict__ tile_meta, int32_t* __restrict__ c_col, V* __restrict__ c_val,
-    i64 c_capacity, int* __restrict__ err) {
+    i64 c_capacity, int* __restrict__ err,
+    const int32_t* __restrict__ s_col_alt = nullptr, const V* __restrict__ s_val_alt = nullptr,  // ALT: the other buffer,
+    const unsigned char* __restrict__ tags = nullptr, u32 alt_bits = 0) {  // the chunks' tags, and which tags live there
   __shared__ int s_rel[kGatherChunkCap + 1];
   __shared__ i64 s_src[kGatherChunkCap];
   __shared__ i64 s_dst[kGatherChunkCap];
@@ -40,6 +46,9 @@ __global__ void __launch_bounds__(kGatherThreads) k7_gather(
       s_rel[i] = (i == n_k) ? tn + 1 : clamp_rel(chunk_nnz_off[k_lo + i] - t0, -(1 << 30), tn + 1);
       if (i < n_k) {
         s_src[i] = chunk_off[k_lo + i];
+        if constexpr (ALT) {
+          if ((alt_bits >> tags[k_lo + i]) & 1u) s_src[i] |= kGatherAltBit;  // (tag 0 never has its bit set)
+        }
         s_dst[i] = chunk_base[k_lo + i];
       }
     }
@@ -70,9 +79,12 @@ __global__ void __launch_bounds__(kGatherThreads) k7_gather(
           if (q < tn) {
             const i64 r = static_cast<i64>(q) - s_rel[k];
             dst[u] = s_dst[k] + r;
-            const i64 src = s_src[k] + r;
-            col[u] = s_col_in[src];
-            val[u] = s_val_in[src];
+            i64 src = s_src[k];
+            bool alt = false;
+            if constexpr (ALT) { alt = (src & kGatherAltBit) != 0; src &= ~kGatherAltBit; }
+            src += r;
+            col[u] = (alt ? s_col_alt : s_col_in)[src];
+            val[u] = (alt ? s_val_alt : s_val_in)[src];
           }
         }
       }
@@ -95,8 +107,10 @@ __global__ void __launch_bounds__(kGatherThreads) k7_gather(
       const i64 r = p - chunk_nnz_off[k];
       const i64 dst = chunk_base[k] + r;
       if (dst < c_capacity) {
-        c_col[dst] = s_col_in[chunk_off[k] + r];
-        c_val[dst] = s_val_in[chunk_off[k] + r];
+        bool alt = false;
+        if constexpr (ALT) alt = (alt_bits >> tags[k]) & 1u;
+        c_col[dst] = (alt ? s_col_alt : s_col_in)[chunk_off[k] + r];
+        c_val[dst] = (alt ? s_val_alt : s_val_in)[chunk_off[k] + r];
       } else {
         dev_set_error(err, kDevCapacity);
       }

@@ -317,6 +317,8 @@ def test_config4_zipf_pair_full_size_default_plan():
     A, B, _ = gen.config_inputs(4)
     info, stats = _check_sampled_rows(A, B, n_random=150, n_heavy=60, whole_row_ptr=True)
     assert info.params.levels() == [256, 2] and info.level0_direct == 0 and info.rows_heavy > 0
+    # after the first split nearly every chunk of these rows is light: the second level moves a fraction of the products
+    assert stats.early_exit_products > 0 and stats.split_products < 2 * stats.staged_products
 
 
 def test_second_workload_class_dense_heavy_rows():
@@ -344,6 +346,7 @@ def test_config4_zipf_wide_columns_three_levels_sampled_rows():
     A, B, _ = gen.config_inputs(4, shrink=2)
     info, stats = _check_sampled_rows(A, B, n_random=60, n_heavy=40, max_fanout=8, chunk_width=8192)
     assert info.params.n_levels == 3 and info.rows_heavy > 0
+    assert stats.early_exit_products > 0  # most chunks of these rows are light after the first split
 
 
 @pytest.mark.parametrize("separate", [0, 1])
@@ -355,6 +358,31 @@ def test_first_level_of_256_children_as_separate_passes(dtype, separate):
     C, info, stats = check_product(A, B, tau=256, chunk_width=1024, separate_histogram=separate, stage_elems=1 << 18)
     assert info.params.levels()[0] == 256 and info.params.n_levels == 2 and info.level0_direct == 0
     assert info.n_batches > 1 and info.rows_heavy > 100
+
+
+@pytest.mark.parametrize("dtype", [np.float32, np.float64])
+@pytest.mark.parametrize("level0", [1, 2])
+@pytest.mark.parametrize("separate", [0, 1])
+def test_light_chunks_leave_the_hierarchy_early(dtype, level0, separate):
+    # Algorithm 3's early exit: from the second level on a chunk with few products is not split further.  Four levels
+    # (fan-out 4, 4, 4, 2), several batches; the same product with every chunk carried through every level must
+    # give the same C, and the multisplit passes must have moved fewer products.
+    A = gen.rmat(13, 16, seed=5, dtype=dtype)
+    common = dict(tau=256, chunk_width=64, max_fanout=4, level0_multisplit=level0, separate_histogram=separate,
+                  stage_elems=1 << 20)
+    C0, info0, st0 = check_product(A, A, early_exit=-1, **common)
+    C1, info1, st1 = check_product(A, A, **common)
+    C2, info2, st2 = check_product(A, A, early_exit=24, **common)
+    assert info1.params.n_levels == 4 and info1.n_batches > 1 and info1.level0_direct == level0 - 1
+    passes = info1.params.n_levels - info1.level0_direct
+    assert st0.early_exit_products == 0 and st0.early_exit_chunks == 0
+    assert st0.split_products == passes * st0.staged_products
+    assert 0 < st2.early_exit_products < st1.early_exit_products <= st1.staged_products
+    assert st1.split_products < st2.split_products < st0.split_products
+    # a chunk leaves at most once, and one that left at level l is moved by l - 1 passes fewer than the rest
+    assert st1.split_products >= passes * st1.staged_products - (info1.params.n_levels - 1) * st1.early_exit_products
+    for C in (C1, C2):
+        assert torch.equal(C.row_ptr, C0.row_ptr) and torch.equal(C.col, C0.col)  # (values: each against the oracle above)
 
 
 @pytest.mark.parametrize("separate", [0, 1])
