@@ -369,8 +369,11 @@ def main():
         ev0.record()
         launches = 0
         stats_sum: dict[str, float] = {}
+        ms_steps = []  # host clock per step (execute returns after a stream synchronize): shows a hiccup if there is one
         for _ in range(steps):
+            t_step = time.perf_counter()
             info, st, nnz = step(True)
+            ms_steps.append(round((time.perf_counter() - t_step) * 1e3, 2))
             launches += int(info.launches + st.launches)
             for name, _t in st._fields_:
                 if name != "reserved":
@@ -390,7 +393,8 @@ def main():
         dom = max(kt, key=lambda k: kt[k]["ms"])
         return {"ms_step": ms_step, "value": replicas_value(products, world, ms_step), "products": products,
                 "info": info, "kernels": kt, "dominant": dom, "launches": launches, "nnz": int(nnz), "clocks": clocks,
-                "early_exit_products": int(stats_avg["early_exit_products"])}
+                "early_exit_products": int(stats_avg["early_exit_products"]), "ms_steps": ms_steps,
+                "ms_execute_device": stats_avg["ms_total"]}
 
     peak, peak_kind = _peaks()
     m = measure(A, B, dA, dB, opts, args.steps, args.warmup, True)
@@ -424,6 +428,7 @@ def main():
                    "early_exit_products": m["early_exit_products"], "plan_opts": args.opt,
                    "step": "gm_spgemm_plan + gm_spgemm_execute (C freed after each step)"},
         "roofline": roofline, "kernels": kt, "clocks": clocks, "gpu_launches": launches,
+        "ms_steps_host_clock": m["ms_steps"], "ms_execute_device": m["ms_execute_device"],
     }
 
     def frac_of(k):
