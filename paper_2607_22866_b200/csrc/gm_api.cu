@@ -619,7 +619,12 @@ static int launch_accumulate(gm_plan* p, const Batch& b, const HeavyBatchState<V
   ++p->stats.launches;
   if (small_max > 0) {
     p->times.begin(PhaseTimes::kAccSmall, st);
-    k6_small_chunks<V><<<static_cast<unsigned>(p->num_sms * 8), kSmallWarps * 32, 0, st>>>(
+    // as many blocks as are resident at once: the warps share out the chunks statically, so a block that had to wait
+    // for a free slot would start its share when the others are done
+    int per_sm = 0;
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, k6_small_chunks<V>, kSmallWarps * 32, 0) != cudaSuccess || per_sm < 1)
+      per_sm = 4;
+    k6_small_chunks<V><<<static_cast<unsigned>(p->num_sms * per_sm), kSmallWarps * 32, 0, st>>>(
         hs.fin_col, hs.fin_val, hs.chunk_off, hs.n_chunks, W, small_max, p->chunk_nnz,
         reinterpret_cast<u64*>(p->c_total + 2), hs.tags, hs.alt_col, hs.alt_val, hs.xt);
     ++p->stats.launches;

@@ -139,6 +139,10 @@ constexpr int kAccSmallChunk = 32 * kSmallMaxPerLane;  // largest chunk the one-
 constexpr int kAccSmallDefault = 256;
 constexpr int kSmallIdxBits = kSmallMaxPerLane == 32 ? 10 : (kSmallMaxPerLane == 16 ? 9 : 8);  // position of a product inside its chunk
 constexpr int kSmallWarps = 4;            // warps per block of the small-chunk kernel
+// Eight blocks per SM: without the bound the compiler takes 105-120 registers and four blocks fit; measured on R-MAT
+// scale 20 fp32 / scale 21 fp64, ms of this kernel with room for 6 / 7 / 8 blocks: 10.0 / 9.9 / 10.1 and
+// 44.0 / 43.6 / 41.6.
+constexpr int kSmallBlocksPerSm = 8;
 
 // Sorts 32 * K packed keys, K per lane, element e = r * 32 + lane in key[r]; ascending in e afterwards.
 // Steps whose partner sits in another lane are the same instruction sequence for every step width, so they run
@@ -194,7 +198,7 @@ __device__ __forceinline__ void warp_sort_keys(u32 (&key)[K], int lane) {
 // One small chunk by one warp.  s_key / s_val: 32 * K entries of this warp's shared memory.
 template <typename V, int K>
 __device__ __forceinline__ int small_chunk(int32_t* col, V* val, int n, u32 wmask, u32* s_key, V* s_val,
-                                           u32* nnz_out, int32_t c_row0, V v_row0) {  // (the caller loaded element `lane`)
+                                           u32* nnz_out) {
   const int lane = threadIdx.x & 31;
   u32 key[K];
   int32_t c_first = 0;
@@ -203,10 +207,10 @@ __device__ __forceinline__ int small_chunk(int32_t* col, V* val, int n, u32 wmas
     const int e = r * 32 + lane;
     key[r] = 0xffffffffu;  // padding sorts to the end
     if (e < n) {
-      const int32_t c = r == 0 ? c_row0 : col[e];
+      const int32_t c = col[e];
       if (e == 0) c_first = c;
       key[r] = ((static_cast<u32>(c) & wmask) << kSmallIdxBits) | static_cast<u32>(e);
-      s_val[e] = r == 0 ? v_row0 : val[e];
+      s_val[e] = val[e];
     }
   }
   const u32 col_base = static_cast<u32>(__shfl_sync(0xffffffffu, c_first, 0)) & ~wmask;
@@ -243,7 +247,7 @@ __device__ __forceinline__ int small_chunk(int32_t* col, V* val, int n, u32 wmas
 }
 
 template <typename V>
-__global__ void __launch_bounds__(kSmallWarps * 32, 8) k6_small_chunks(
+__global__ void __launch_bounds__(kSmallWarps * 32, kSmallBlocksPerSm) k6_small_chunks(
     int32_t* x_col, V* x_val, const i64* __restrict__ chunk_off, i64 n_chunks, int W, int small_max,
     u32* __restrict__ chunk_nnz,
     u64* __restrict__ totals,  // [0] += products, [1] += entries of the chunks handled here (statistics)
@@ -267,51 +271,28 @@ __global__ void __launch_bounds__(kSmallWarps * 32, 8) k6_small_chunks(
       if (tags) ctag = tags[k];
     }
     u32 todo = __ballot_sync(0xffffffffu, cn > 0 && cn <= small_max);
-    if (!todo) continue;
-    // A chunk's work starts with a round trip to HBM and the warp has nothing else to do meanwhile, so the first 32
-    // products of the next chunk are requested before the current chunk is sorted (most small chunks hold no more).
-    struct Job {
-      int32_t* col;
-      V* val;
-      int n, src;
-      u32 wm;
-      int32_t c0;
-      V v0;
-    };
-    auto open_job = [&](int src) {
-      Job j;
+    // (Requesting the next chunk's first products before the current chunk is sorted was tried: no gain at 64
+    // registers, and the extra live state spilled in the fp64 kernel, 42 -> 60 ms on R-MAT scale 21.)
+    while (todo) {
+      const int src = __ffs(todo) - 1;
+      todo &= todo - 1;
       const i64 s0 = __shfl_sync(0xffffffffu, cs, src);
-      j.n = __shfl_sync(0xffffffffu, cn, src);
-      j.src = src;
+      const int n = __shfl_sync(0xffffffffu, cn, src);
       const int tag = __shfl_sync(0xffffffffu, ctag, src);
       // an early chunk lies in the buffer it was left in and is sorted over all the columns it spans
       const bool alt = tag && xt.alt(tag);
-      j.col = (alt ? x_col_alt : x_col) + s0;
-      j.val = (alt ? x_val_alt : x_val) + s0;
-      j.wm = tag ? (1u << xt.span_bits(tag)) - 1u : wmask;
-      j.c0 = 0;
-      j.v0 = V(0);
-      if (lane < j.n) { j.c0 = j.col[lane]; j.v0 = j.val[lane]; }
-      return j;
-    };
-    Job cur = open_job(__ffs(todo) - 1);
-    todo &= todo - 1;
-    for (;;) {
-      const bool more = todo != 0;  // (uniform)
-      Job nxt = cur;
-      if (more) { nxt = open_job(__ffs(todo) - 1); todo &= todo - 1; }
-      const int n = cur.n;
-      u32* out = &chunk_nnz[(g << 5) + cur.src];
+      int32_t* col = (alt ? x_col_alt : x_col) + s0;
+      V* val = (alt ? x_val_alt : x_val) + s0;
+      const u32 wm = tag ? (1u << xt.span_bits(tag)) - 1u : wmask;
+      u32* out = &chunk_nnz[(g << 5) + src];
       int m;
-      if (n <= 32) m = small_chunk<V, 1>(cur.col, cur.val, n, cur.wm, s_key[w], s_val[w], out, cur.c0, cur.v0);
-      else if (n <= 64) m = small_chunk<V, 2>(cur.col, cur.val, n, cur.wm, s_key[w], s_val[w], out, cur.c0, cur.v0);
-      else if (n <= 128) m = small_chunk<V, 4>(cur.col, cur.val, n, cur.wm, s_key[w], s_val[w], out, cur.c0, cur.v0);
-      else if (kSmallMaxPerLane == 8 || n <= 256) m = small_chunk<V, 8>(cur.col, cur.val, n, cur.wm, s_key[w], s_val[w], out, cur.c0, cur.v0);
-      else if (kSmallMaxPerLane == 16 || n <= 512) m = small_chunk<V, (kSmallMaxPerLane >= 16 ? 16 : 8)>(cur.col, cur.val, n, cur.wm, s_key[w], s_val[w], out, cur.c0, cur.v0);
-      else m = small_chunk<V, kSmallMaxPerLane>(cur.col, cur.val, n, cur.wm, s_key[w], s_val[w], out, cur.c0, cur.v0);
+      if (n <= 32) m = small_chunk<V, 1>(col, val, n, wm, s_key[w], s_val[w], out);
+      else if (n <= 64) m = small_chunk<V, 2>(col, val, n, wm, s_key[w], s_val[w], out);
+      else if (n <= 128) m = small_chunk<V, 4>(col, val, n, wm, s_key[w], s_val[w], out);
+      else if (kSmallMaxPerLane == 8 || n <= 256) m = small_chunk<V, 8>(col, val, n, wm, s_key[w], s_val[w], out);
+      else if (kSmallMaxPerLane == 16 || n <= 512) m = small_chunk<V, (kSmallMaxPerLane >= 16 ? 16 : 8)>(col, val, n, wm, s_key[w], s_val[w], out);
+      else m = small_chunk<V, kSmallMaxPerLane>(col, val, n, wm, s_key[w], s_val[w], out);
       if (lane == 0) { s_sum[w][0] += static_cast<u64>(n); s_sum[w][1] += static_cast<u64>(m); }
-      if (!more) break;
-      cur = nxt;
     }
   }
   if (lane == 0 && s_sum[w][0]) {
