@@ -88,8 +88,8 @@ class ClockSampler:
               "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
               "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
 
-    def __init__(self, gpu_index: int):
-        self.gpu_index, self.proc, self.path = gpu_index, None, None
+    def __init__(self, gpu_index: int, interval: float = 0.2):
+        self.gpu_index, self.proc, self.path, self.interval = gpu_index, None, None, interval
         self.thread, self.stop_flag, self.sm, self.mx, self.reasons = None, False, [], [], set()
 
     def _nvml_loop(self, nv, handle):
@@ -109,7 +109,7 @@ class ClockSampler:
                         self.reasons.add(name)
             except Exception:
                 pass
-            time.sleep(0.2)
+            time.sleep(self.interval)
 
     def start(self):
         try:
@@ -296,6 +296,8 @@ def main():
     ap.add_argument("--cpu-budget", type=float, default=15.0, help="seconds of oracle time for the CPU baseline")
     ap.add_argument("--e2e-steps", type=int, default=2)
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--clock-interval", type=float, default=0.2,
+                    help="seconds between clock samples during the timed region (0: no sampling; diagnostic)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-extra", action="store_true",
                     help="skip the forced-multisplit step and the per-config list (default workload only)")
@@ -346,22 +348,28 @@ def main():
         """`warmup` untimed and `steps` timed products (plan + execute each).  Returns a dict with the step time,
         the plan's facts, the per-kernel table (algorithmic bytes, CUDA-event time) and the dominant kernel."""
         sv = A.val.dtype.itemsize
+        step_parts = []
 
         def step(timing: bool):
+            t_a = time.perf_counter()
             plan = gm.spgemm_plan(dA, dB, SMEM_BYTES, opts)
+            t_b = time.perf_counter()
             if timing:
                 plan.set_timing(True)
             C = gm.spgemm_execute(plan)
+            t_c = time.perf_counter()
             info, st = plan.info(), plan.stats()
             nnz = C.nnz
             del C
             plan.destroy()
+            if timing:  # host clock: plan, execute (both return after a stream synchronize); device: execute
+                step_parts.append([round((t_b - t_a) * 1e3, 2), round((t_c - t_b) * 1e3, 2), round(float(st.ms_total), 2)])
             return info, st, nnz
 
         for _ in range(warmup):
             info, st, nnz = step(False)
         barrier()
-        sampler = ClockSampler(local_rank) if sample_clocks else None
+        sampler = ClockSampler(local_rank, args.clock_interval) if sample_clocks and args.clock_interval > 0 else None
         if sampler:
             sampler.start()
         ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
@@ -393,7 +401,7 @@ def main():
         dom = max(kt, key=lambda k: kt[k]["ms"])
         return {"ms_step": ms_step, "value": replicas_value(products, world, ms_step), "products": products,
                 "info": info, "kernels": kt, "dominant": dom, "launches": launches, "nnz": int(nnz), "clocks": clocks,
-                "early_exit_products": int(stats_avg["early_exit_products"]), "ms_steps": ms_steps,
+                "early_exit_products": int(stats_avg["early_exit_products"]), "ms_steps": ms_steps, "step_parts": step_parts,
                 "ms_execute_device": stats_avg["ms_total"]}
 
     peak, peak_kind = _peaks()
@@ -429,6 +437,7 @@ def main():
                    "step": "gm_spgemm_plan + gm_spgemm_execute (C freed after each step)"},
         "roofline": roofline, "kernels": kt, "clocks": clocks, "gpu_launches": launches,
         "ms_steps_host_clock": m["ms_steps"], "ms_execute_device": m["ms_execute_device"],
+        "ms_plan_execute_host_execute_device": m["step_parts"],
     }
 
     def frac_of(k):
