@@ -12,16 +12,20 @@
 namespace gm {
 
 constexpr int kGatherThreads = 256;
-constexpr int kGatherTile = 4096;
-#ifndef GM_GATHER_BATCH
-#define GM_GATHER_BATCH 6
-#endif
-// rows a warp has in flight.  The kernel is bound by bytes in flight (fp32 moved 4.3 TB/s where fp64, with twice the
-// bytes per load, moved 6.1): measured 36.0 / 32.3 / 34.9 ms per step on R-MAT scale 20 with 4 / 6 / 8.
-constexpr int kGatherBatch = GM_GATHER_BATCH;
+// Output positions per block.  Measured on R-MAT scale 20 fp32 (ms per step of this kernel) with 2048 / 4096 / 8192 /
+// 16384: 33.6 / 30.2 / 28.9 / 28.6; the clipped-Zipf pair, whose chunks hold a few entries each, prefers 8192 to 16384
+// (0.95 against 1.18 ms: fewer tiles with more chunks than the shared table holds).
+constexpr int kGatherTile = 8192;
+// Rows of 64 positions a warp has in flight.  With 4-byte accesses and rows of 32 the kernel wanted six in flight
+// (36.0 / 32.3 / 34.9 ms with 4 / 6 / 8); with paired accesses one row of 64 is best (30.2 / 30.5 / 35.3 / 38.7 ms with
+// 1 / 2 / 3 / 4 at 4096 positions per block: registers cost occupancy).
+constexpr int kGatherBatch = 1;
 constexpr int kGatherChunkCap = 1024;  // chunks staged in shared memory per tile; more -> per-element search
 
 constexpr i64 kGatherAltBit = i64{1} << 62;
+template <typename V> struct Pair;
+template <> struct Pair<float> { using type = float2; };
+template <> struct Pair<double> { using type = double2; };
 
 template <typename V, bool ALT = false>
 __global__ void __launch_bounds__(kGatherThreads) k7_gather(
@@ -53,50 +57,83 @@ __global__ void __launch_bounds__(kGatherThreads) k7_gather(
       }
     }
     __syncthreads();
-    // A warp takes rows of 32 consecutive positions (row w, w + 8, ...), kGatherBatch rows at a time with all loads
-    // before the first store.  Chunks hold hundreds of entries on average, so a row usually lies inside one chunk:
-    // the warp keeps a uniform chunk cursor, and only a row that crosses a chunk boundary lets its lanes step on
-    // from there (the per-position binary search this replaces cost more instructions than the copy itself).
+    // A warp takes rows of 64 consecutive positions, kGatherBatch rows at a time with all loads before the first
+    // store.  Chunks hold hundreds of entries on average, so a row usually lies inside one chunk (the warp keeps a
+    // uniform chunk cursor); then every lane copies two neighbouring entries with one 8-byte load per array (16-byte
+    // for fp64 values): the kernel is bound by the bytes it has in flight, and a load instruction then carries twice
+    // as many.  If the row's source starts at an odd index the pairs start one entry early, and lane 0, whose first
+    // entry is not the row's, fetches the row's last one instead.  A row that crosses a chunk boundary lets every lane
+    // find the chunks of its two positions from the cursor on.
     constexpr int kWarps = kGatherThreads / 32;
+    constexpr int kRow = 64;
+    using V2 = typename Pair<V>::type;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     int cur = 0;  // warp-uniform: last chunk whose start is <= the row's first position
-    for (int r0 = warp * 32; r0 < tn; r0 += kGatherBatch * kWarps * 32) {
-      i64 dst[kGatherBatch];
-      int32_t col[kGatherBatch];
-      V val[kGatherBatch];
+    for (int r0 = warp * kRow; r0 < tn; r0 += kGatherBatch * kWarps * kRow) {
+      i64 d0[kGatherBatch], d1[kGatherBatch];  // where the lane's two entries go (-1: nothing)
+      int32_t c0[kGatherBatch], c1[kGatherBatch];
+      V v0[kGatherBatch], v1[kGatherBatch];
 #pragma unroll
       for (int u = 0; u < kGatherBatch; ++u) {
-        const int q0 = r0 + u * kWarps * 32;
-        const int q = q0 + lane;
-        dst[u] = -1;
+        const int q0 = r0 + u * kWarps * kRow;
+        d0[u] = -1;
+        d1[u] = -1;
         if (q0 < tn) {  // (uniform)
           while (s_rel[cur + 1] <= q0) ++cur;  // empty chunks share a start with their successor and are skipped
-          int k = cur;
-          if (s_rel[cur + 1] < q0 + 32) {      // the row crosses into later chunks
-            if (q < tn)
-              while (s_rel[k + 1] <= q) ++k;
-          }
-          if (q < tn) {
-            const i64 r = static_cast<i64>(q) - s_rel[k];
-            dst[u] = s_dst[k] + r;
-            i64 src = s_src[k];
+          if (q0 + kRow <= min(s_rel[cur + 1], tn)) {
+            i64 src = s_src[cur];
             bool alt = false;
             if constexpr (ALT) { alt = (src & kGatherAltBit) != 0; src &= ~kGatherAltBit; }
-            src += r;
-            col[u] = (alt ? s_col_alt : s_col_in)[src];
-            val[u] = (alt ? s_val_alt : s_val_in)[src];
+            const int32_t* const colp = alt ? s_col_alt : s_col_in;
+            const V* const valp = alt ? s_val_alt : s_val_in;
+            const i64 off = static_cast<i64>(q0) - s_rel[cur];
+            const i64 src0 = src + off, dst0 = s_dst[cur] + off;
+            const i64 odd = src0 & 1;
+            const i64 a = src0 - odd + 2 * lane;  // even: the pair is naturally aligned
+            const int2 cc = *reinterpret_cast<const int2*>(colp + a);
+            const V2 vv = *reinterpret_cast<const V2*>(valp + a);
+            c0[u] = cc.x; c1[u] = cc.y;
+            v0[u] = vv.x; v1[u] = vv.y;
+            d0[u] = dst0 - odd + 2 * lane;
+            d1[u] = d0[u] + 1;
+            if (odd && lane == 0) {
+              c0[u] = colp[src0 + kRow - 1];
+              v0[u] = valp[src0 + kRow - 1];
+              d0[u] = dst0 + kRow - 1;
+            }
+          } else {
+#pragma unroll
+            for (int h = 0; h < 2; ++h) {
+              const int q = q0 + h * 32 + lane;
+              if (q < tn) {
+                int k = cur;
+                while (s_rel[k + 1] <= q) ++k;
+                const i64 r = static_cast<i64>(q) - s_rel[k];
+                i64 src = s_src[k];
+                bool alt = false;
+                if constexpr (ALT) { alt = (src & kGatherAltBit) != 0; src &= ~kGatherAltBit; }
+                src += r;
+                const int32_t c = (alt ? s_col_alt : s_col_in)[src];
+                const V v = (alt ? s_val_alt : s_val_in)[src];
+                if (h == 0) { c0[u] = c; v0[u] = v; d0[u] = s_dst[k] + r; }
+                else { c1[u] = c; v1[u] = v; d1[u] = s_dst[k] + r; }
+              }
+            }
           }
         }
       }
 #pragma unroll
       for (int u = 0; u < kGatherBatch; ++u) {
-        if (dst[u] >= 0) {
-          if (dst[u] < c_capacity) {
-            c_col[dst[u]] = col[u];
-            c_val[dst[u]] = val[u];
-          } else {
-            dev_set_error(err, kDevCapacity);
-          }
+        if (max(d0[u], d1[u]) >= c_capacity) {
+          dev_set_error(err, kDevCapacity);
+        } else if (d0[u] >= 0 && d1[u] == d0[u] + 1 && !(d0[u] & 1)) {
+          *reinterpret_cast<int2*>(c_col + d0[u]) = make_int2(c0[u], c1[u]);
+          V2 vv;
+          vv.x = v0[u]; vv.y = v1[u];
+          *reinterpret_cast<V2*>(c_val + d0[u]) = vv;
+        } else {
+          if (d0[u] >= 0) { c_col[d0[u]] = c0[u]; c_val[d0[u]] = v0[u]; }
+          if (d1[u] >= 0) { c_col[d1[u]] = c1[u]; c_val[d1[u]] = v1[u]; }
         }
       }
     }
