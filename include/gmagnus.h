@@ -165,7 +165,8 @@ typedef struct gm_exec_stats {
 
 typedef struct gm_plan gm_plan; /* opaque, owned by the library */
 
-/* Device allocator hook.  alloc(bytes, stream, user) returns a device pointer or NULL; it is
+/* Device allocator hook.  alloc(bytes, stream, user) returns a device pointer aligned to at least
+ * 256 bytes (the kernels use 16-byte accesses into the workspace and into C), or NULL; it is
  * called from host code of plan/execute only, never from a kernel.  Passing NULLs restores the
  * default (stream-ordered cudaMallocAsync on the device's default pool). */
 typedef void* (*gm_alloc_fn)(size_t bytes, void* cuda_stream, void* user);

@@ -76,7 +76,17 @@ static void* default_alloc(size_t bytes, cudaStream_t st) {
 
 static void* dev_alloc(size_t bytes, cudaStream_t st) {
   if (bytes == 0) bytes = 16;
-  if (g_alloc.alloc) return g_alloc.alloc(bytes, st, g_alloc.user);
+  if (g_alloc.alloc) {
+    void* p = g_alloc.alloc(bytes, st, g_alloc.user);
+    // the kernels use 16-byte accesses into what they are given: a hook that hands out less aligned memory is
+    // treated like one that has none
+    if (p && reinterpret_cast<uintptr_t>(p) % 256 != 0) {
+      if (g_alloc.free) g_alloc.free(p, st, g_alloc.user);
+      fail(GM_ERR_OOM, "the allocator hook returned a pointer that is not 256-byte aligned");
+      return nullptr;
+    }
+    return p;
+  }
   return default_alloc(bytes, st);
 }
 static void dev_free(void* p, cudaStream_t st) {

@@ -261,6 +261,25 @@ def test_host_entry_point_streams_batches_to_the_host(dtype):
     assert ei.value.status == -6
 
 
+def test_host_entry_point_with_chunks_that_left_the_hierarchy_early():
+    # three levels with early exit, several batches, result streamed to the host: the gather reads the chunks that
+    # stayed behind from the other staging buffer
+    import paper_2607_22866_b200 as gm
+    A = gen.rmat(12, 16, seed=21, dtype=np.float32)
+    ref = oracle.spgemm(A, A)
+    o = gm.PlanOpts()
+    o.tau, o.chunk_width, o.max_fanout, o.stage_elems, o.validate_inputs = 128, 128, 4, 1 << 18, 1
+    rp = np.empty(A.n_rows + 1, np.int64)
+    col = np.empty(ref.nnz, np.int32)
+    val = np.empty(ref.nnz, np.float32)
+    nnz = gm.spgemm_host(A, A, rp, col, val, opts=o)
+    assert nnz == ref.nnz and np.array_equal(rp, ref.row_ptr) and np.array_equal(col, ref.col)
+    assert np.all(np.abs(val.astype(np.float64) - ref.val) <= 1e-5 * ref.abs)
+    dA = gm.DeviceCSR.from_host(A)
+    C, info, stats = gm.spgemm(dA, dA, 232448, o)
+    assert info.params.n_levels == 3 and info.n_batches > 1 and stats.early_exit_products > 0
+
+
 def _check_sampled_rows(A, B, n_random=200, n_heavy=60, whole_row_ptr=False, **opts):
     """Full-size check in the launch configuration the benchmark times: structure and values of
     sampled rows (random rows, the heaviest rows, random heavy rows) against the row-range oracle,
