@@ -84,7 +84,7 @@ typedef struct gm_plan_opts {
                               the first level's children itself; 0 (default) = the latter when the heavy
                               rows' segments are long compared with the fan-out, else the former        */
   int32_t small_chunk_max; /* final chunks of at most this many products are sorted by one warp each (Section
-                              III-A's branch for light chunks); 0 = default (256), -1 = none, at most 512        */
+                              III-A's branch for light chunks); 0 = default (128), -1 = none, at most 512        */
   int32_t mid_chunk_max;   /* final chunks of at most this many products (and more than small_chunk_max) get one
                               128-thread block each, symbolic then numeric pass over a compact array; larger
                               ones go to the dense W-column accumulator.  0 = default (4096 for fp32, 2048 for

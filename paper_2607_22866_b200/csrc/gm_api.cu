@@ -225,6 +225,9 @@ struct gm_plan {
   cudaEvent_t ev_fork = nullptr, ev_light = nullptr;
 };
 
+#ifndef GM_MID_MIN_BLOCKS
+#define GM_MID_MIN_BLOCKS 7
+#endif
 namespace gm {
 
 template <typename T>
@@ -302,7 +305,8 @@ static int build_plan(gm_plan* p, cudaStream_t st) {
     p->small_max = o.small_chunk_max < 0 ? 0 : (o.small_chunk_max ? o.small_chunk_max : kAccSmallDefault);
     int mid = o.mid_chunk_max < 0 ? 0 : (o.mid_chunk_max ? o.mid_chunk_max : (p->sv == 4 ? 4096 : 2048));
     // several mid-chunk blocks must fit an SM next to each other for the class to pay
-    while (mid > p->small_max && mid_smem_bytes(prm.chunk_width, p->sv, mid) + 1024 > p->smem_bytes / 8) mid /= 2;
+    while (mid > p->small_max && mid_smem_bytes(prm.chunk_width, p->sv, mid) + 1024 > p->smem_bytes / GM_MID_MIN_BLOCKS) mid /= 2;
+    if (prm.chunk_width > 65536) mid = 0;  // the kernel keeps a chunk's columns as 16-bit offsets
     p->mid_max = std::max(mid, p->small_max);
     if (o.early_exit < -1 || o.early_exit > kAccSmallChunk) return fail(GM_ERR_INVALID_ARG, "early_exit out of range");
     // early exit needs the one-warp sort (the only accumulate kernel that takes a chunk wider than W) and a level

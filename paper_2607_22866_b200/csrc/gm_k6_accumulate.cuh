@@ -134,9 +134,9 @@ __global__ void k6_chunk_bases(const i64* __restrict__ chunk_nnz_off, i64 n_chun
 constexpr int kSmallMaxPerLane = GM_SMALL_PER_LANE;
 constexpr int kAccSmallChunk = 32 * kSmallMaxPerLane;  // largest chunk the one-warp sort can take
 // Default hand-over to the mid-size kernel.  The sort costs n log^2 n; measured on B200 (R-MAT scale 20 fp32 / scale 21
-// fp64, small + mid kernels together): 55 / 105 ms with chunks up to 512 products sorted, 50 / 90 ms up to 256,
-// 53 / 99 ms up to 128.
-constexpr int kAccSmallDefault = 256;
+// fp64, small + mid kernels together, ms per step) with chunks up to 64 / 96 / 128 / 192 / 256 products sorted:
+// 42.4 / 41.4 / 41.0 / 41.1 / 42.8 and 81.7 / 77.4 / 75.2 / 75.5 / 76.5.
+constexpr int kAccSmallDefault = 128;
 constexpr int kSmallIdxBits = kSmallMaxPerLane == 32 ? 10 : (kSmallMaxPerLane == 16 ? 9 : 8);  // position of a product inside its chunk
 constexpr int kSmallWarps = 4;            // warps per block of the small-chunk kernel
 // Eight blocks per SM: without the bound the compiler takes 105-120 registers and four blocks fit; measured on R-MAT
@@ -305,7 +305,8 @@ __global__ void __launch_bounds__(kSmallWarps * 32, kSmallBlocksPerSm) k6_small_
 // ---------------------------------------------------------------------------------------------------------
 // Mid-size chunks: one block of kMidThreads threads per chunk, symbolic pass then numeric pass.
 // Shared memory: bitmap (W/32 words) | rank of every word's first entry (16 bits each) | the chunk's values,
-// compact (mid_max entries).  A thread owns consecutive bitmap words and moves them with 16-byte accesses.
+// compact (mid_max entries) | the chunk's columns, compact (16 bits each: W <= 65536).  In the scan a thread owns
+// consecutive bitmap words and moves them with 16-byte accesses.
 // ---------------------------------------------------------------------------------------------------------
 // Products a thread holds per tile.  The unrolled slots are executed whether a chunk fills them or not, and most
 // chunks of this class are small: measured on R-MAT scale 20 fp32 / scale 21 fp64, ms per step of this kernel with
@@ -315,7 +316,7 @@ constexpr int kMidTile = kMidThreads * kMidPer;     // 512: chunks up to this si
 
 inline size_t mid_smem_bytes(int W, int val_bytes, int mid_max) {
   const size_t n_words = static_cast<size_t>(W) / 32;
-  return ((n_words * 6 + 15) & ~size_t{15}) + static_cast<size_t>(mid_max) * val_bytes + 64;
+  return ((n_words * 6 + 15) & ~size_t{15}) + static_cast<size_t>(mid_max) * (val_bytes + 2) + 64;
 }
 
 struct ChunkTask {
@@ -380,6 +381,7 @@ __global__ void __launch_bounds__(kMidThreads) k6_mid_chunks(
   u32* bitmap = reinterpret_cast<u32*>(smem_mid_raw);                 // n_words
   unsigned short* wpre = reinterpret_cast<unsigned short*>(bitmap + n_words);  // n_words: rank of the word's first entry
   V* oval = reinterpret_cast<V*>(smem_mid_raw + ((static_cast<size_t>(n_words) * 6 + 15) & ~size_t{15}));
+  unsigned short* ocol = reinterpret_cast<unsigned short*>(oval + mid_max);  // the entries' columns inside the chunk
   __shared__ u32 s_wsum[T / 32];
   __shared__ ChunkTask s_task[2];
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -478,6 +480,7 @@ __global__ void __launch_bounds__(kMidThreads) k6_mid_chunks(
         if (c != 0xffffffffu) {
           const u32 r = static_cast<u32>(wpre[c >> 5]) + __popc(bitmap[c >> 5] & ((1u << (c & 31)) - 1u));
           atomicAdd(&oval[r], v_reg[u]);
+          ocol[r] = static_cast<unsigned short>(c);  // (every product of the column writes the same value)
         }
       }
       if (++tile >= n_tiles) break;
@@ -493,33 +496,21 @@ __global__ void __launch_bounds__(kMidThreads) k6_mid_chunks(
     // the next chunk's first columns are requested before this chunk is written out
     const ChunkTask next = s_task[par ^ 1];
     if (next.k >= 0) load_cols(next, 0);
-    // ---- write-out in place: columns from the bitmap (each thread its own words), values from the compact array
-    if (own && pc) {
-      u32 p = ex;
-      auto emit_word = [&](u32 bits, int w) {
-        const u32 cb = col_base + (static_cast<u32>(w) << 5);
-        while (bits) {
-          const int b = __ffs(bits) - 1;
-          bits &= bits - 1;
-          col[p++] = static_cast<int32_t>(cb + b);
-        }
-      };
-      if (wpt == 8) {
-        emit_word(b0.x, wb); emit_word(b0.y, wb + 1); emit_word(b0.z, wb + 2); emit_word(b0.w, wb + 3);
-        emit_word(b1.x, wb + 4); emit_word(b1.y, wb + 5); emit_word(b1.z, wb + 6); emit_word(b1.w, wb + 7);
-        *reinterpret_cast<uint4*>(bitmap + wb) = make_uint4(0, 0, 0, 0);
-        *reinterpret_cast<uint4*>(bitmap + wb + 4) = make_uint4(0, 0, 0, 0);
-      } else {
-        for (int i = 0; i < wpt; ++i) {
-          const u32 bits = bitmap[wb + i];
-          if (bits) {
-            bitmap[wb + i] = 0u;
-            emit_word(bits, wb + i);
-          }
-        }
-      }
+    // ---- write-out in place: columns from the bitmap, values from the compact array.  The words are dealt out
+    // round-robin here, not in the runs of the scan: the dense words of a power-law chunk are its first ones (hub
+    // columns), and one thread writing all their columns held the block up (cycle counters on R-MAT scale 20: 10.5 k
+    // of thread 0's 21 k cycles per chunk were this loop, 6 k of the last thread's).
+    // ---- write-out in place, from the compact arrays: position i of the chunk's result takes column ocol[i] and
+    // value oval[i], so the copy is coalesced and the same for every thread.  (Walking the bitmap instead, each
+    // thread the columns of its own words, took 37.4 ms on R-MAT scale 20 where this takes 32.7: the dense words
+    // of a power-law chunk are its first ones, and their owners' serial loops were most of the kernel's instructions.)
+    if ((n_words & 3) == 0) {
+      for (int w = tid * 4; w < n_words; w += T * 4) *reinterpret_cast<uint4*>(bitmap + w) = make_uint4(0, 0, 0, 0);
+    } else {
+      for (int w = tid; w < n_words; w += T) bitmap[w] = 0u;
     }
     for (int i = tid; i < static_cast<int>(total); i += T) {
+      col[i] = static_cast<int32_t>(col_base + ocol[i]);
       val[i] = oval[i];
       oval[i] = V(0);
     }
