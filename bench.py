@@ -43,7 +43,7 @@ DEFAULT_CONFIG = 2  # R-MAT scale 20, edge factor 16, fp32: the largest fp32 pow
 # (R-MAT scale 17: one batch holds the whole product, 1.09 G products, about 9 GB staged).  Traffic grows in
 # proportion to the products processed, so a full-size launch is its algorithmic figure times this ratio.  A kernel
 # that has changed since its capture must lose its entry (traffic is then reported as null).
-TRAFFIC_RATIO = {"k4_expand": 1.04, "k5a_histogram": 1.00, "k5b_multisplit": 1.00, "k6_small_chunks": 0.66,
+TRAFFIC_RATIO = {"k4_expand": 1.03, "k5a_histogram": 1.00, "k5b_multisplit": 1.00, "k6_small_chunks": 0.63,
                  "k6_mid_chunks": 0.99, "k6_accumulate": 1.00, "k7_gather": 1.00}
 TRAFFIC_SOURCE = ("single-kernel, single-launch ncu DRAM-counter captures on the same recipe 2**3 smaller (R-MAT scale 17, "
                   "one batch holds the whole product), scaled by products")
