@@ -516,3 +516,43 @@ def test_chunk_sizes_around_the_warp_sort_widths(dtype):
     assert chunk1.min() == 1 and (chunk1 > 512).any() and {32, 33, 256, 257}.issubset(set(chunk1.tolist()))
     C, info, stats = check_product(A, B, tau=1, chunk_width=1024, max_fanout=4)
     assert info.rows_heavy == int((chunk1 + patA.sum(axis=1) > 1).sum())
+
+
+@pytest.mark.parametrize("seed", list(range(48)))
+def test_random_plans_against_the_oracle(seed):
+    # seeded draws of matrix shape and of every plan option that changes how the work is split: whatever the split,
+    # C must be the oracle's (debug validation on: inputs checked, every product checked against its chunk)
+    rng = np.random.default_rng(1000 + seed)
+    dtype = [np.float32, np.float64][seed % 2]
+    kind = seed % 3
+    if kind == 0:
+        A = gen.rmat(int(rng.integers(9, 13)), int(rng.integers(4, 20)), seed=100 + seed, dtype=dtype)
+        B = A
+    elif kind == 1:
+        m = int(rng.integers(300, 2000))
+        A = random_csr(rng, int(rng.integers(20, 400)), m, float(rng.uniform(0.01, 0.3)), dtype)
+        B = random_csr(rng, m, int(rng.integers(100, 5000)), float(rng.uniform(0.002, 0.05)), dtype,
+                       zero_fraction=0.05)
+    else:
+        A = gen.zipf_rows(int(rng.integers(200, 3000)), 4000, 1.6, 600, seed=200 + seed, dtype=dtype)
+        B = gen.zipf_rows(4000, int(rng.integers(500, 200000)), 1.8, 300, seed=300 + seed, dtype=dtype)
+    opts = dict(
+        tau=int(rng.choice([8, 32, 128, 512])),
+        chunk_width=int(rng.choice([32, 64, 256, 1024, 4096])),
+        max_fanout=int(rng.choice([2, 4, 16, 256])),
+        stage_elems=int(rng.choice([0, 1 << 16, 1 << 19])),
+        level0_multisplit=int(rng.integers(0, 3)),
+        separate_histogram=int(rng.integers(0, 2)),
+        early_exit=int(rng.choice([0, -1, 16])),
+        small_chunk_max=int(rng.choice([0, 32, 512, -1])),
+        mid_chunk_max=int(rng.choice([0, 64, 1024, -1])),
+        expand_order=int(rng.choice([0, 0, 1])),
+        single_stream=int(rng.integers(0, 2)),
+        acc_ctas_per_sm=int(rng.choice([1, 2, 4])),
+    )
+    ip = oracle.row_products(A, B)
+    if opts["stage_elems"]:
+        opts["stage_elems"] = max(opts["stage_elems"], int(ip.max()))
+    while opts["max_fanout"] ** 8 < -(-B.n_cols // opts["chunk_width"]):  # the split may take at most eight levels
+        opts["max_fanout"] *= 4
+    check_product(A, B, **opts)
