@@ -496,7 +496,7 @@ static int build_plan(gm_plan* p, cudaStream_t st) {
       GM_TRY(plan_alloc(p, &p->exit_tag[1], n_chunks_max + 1, st));
       GM_TRY(plan_alloc(p, &p->parent_tag, n_chunks_max + 1, st));
     }
-    const size_t n_tiles_max = static_cast<size_t>(info.stage_elems) / std::min({kExpandTile, kSplitTile, kGatherTile, kDirectTile}) + 2;
+    const size_t n_tiles_max = static_cast<size_t>(info.stage_elems) / std::min({kExpandTile, kSplitTile, kGatherTile, kDirectTileSmall}) + 2;
     GM_TRY(plan_alloc(p, &p->tile_meta, n_tiles_max, st));
     GM_TRY(plan_alloc(p, &p->row_meta, n_tiles_max, st));
     if (p->direct) {
@@ -767,11 +767,12 @@ static int heavy_batch_front(gm_plan* p, const Batch& b, HeavyBatchState<V>* hs,
           p->seg_off, p->seg_bstart, p->B.col_idx, static_cast<const V*>(p->B.vals), seg0, n_seg_b, p->seg_rec, F, prm.shift[0],
           p->stage_col[0], static_cast<V*>(p->stage_val[0]));
     } else {
-      const unsigned grid = static_cast<unsigned>((b.elems + kDirectTile - 1) / kDirectTile);
-      k_tile_bounds<<<grid_for(grid, 256, p->num_sms), 256, 0, st>>>(p->seg_off, p->n_seg, b.elem0, b.elems, kDirectTile,
-                                                                   p->tile_meta);
-      k_tile_bounds<<<grid_for(grid, 256, p->num_sms), 256, 0, st>>>(off_cur, rows_b, 0, b.elems, kDirectTile, p->row_meta);
-      k4_expand_direct<V><<<grid, kExpandThreads, 0, st>>>(
+      const int tile = direct_tile(F);
+      const unsigned grid = static_cast<unsigned>((b.elems + tile - 1) / tile);
+      k_tile_bounds<<<grid_for(grid, 256, p->num_sms), 256, 0, st>>>(p->seg_off, p->n_seg, b.elem0, b.elems, tile, p->tile_meta);
+      k_tile_bounds<<<grid_for(grid, 256, p->num_sms), 256, 0, st>>>(off_cur, rows_b, 0, b.elems, tile, p->row_meta);
+      auto kern = tile == kDirectTileSmall ? k4_expand_direct<V, kDirectTileSmall> : k4_expand_direct<V, kExpandTile>;
+      kern<<<grid, kExpandThreads, 0, st>>>(
           p->seg_off, p->seg_bstart, p->seg_j, p->tile_meta, static_cast<const V*>(p->A.vals), p->B.col_idx,
           static_cast<const V*>(p->B.vals), b.elem0, b.elems, p->row_meta, off_cur, seg0, F, prm.shift[0], row_base, p->seg_h,
           p->stage_col[0], static_cast<V*>(p->stage_val[0]));

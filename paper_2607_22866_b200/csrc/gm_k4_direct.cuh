@@ -119,11 +119,14 @@ __global__ void k_g_row_base(const u32* __restrict__ G, const i64* __restrict__ 
   }
 }
 
-// Products per block.  A smaller tile than the row-order expansion's: more tiles then have few enough (segment, child)
-// pairs for the shared table of run starts.  Measured, ms per step of this kernel with 2048 / 4096 / 8192 / 16384:
-// R-MAT scale 20 fp32 (32 children) 71.9 / 60.3 / 61.7 / 67.4, R-MAT scale 21 fp64 (128 children) 80.5 / 72.5 / 77.9 / -.
-constexpr int kDirectTile = 4096;
-template <typename V>
+// Products per block: the row-order expansion's 8192 for a first level of few children, half of that from 32
+// children on.  Measured, ms per step of this kernel with 2048 / 4096 / 8192 / 16384: R-MAT scale 20 fp32 (32 children)
+// 71.9 / 60.3 / 61.7 / 67.4, R-MAT scale 21 fp64 (128 children) 80.5 / 72.5 / 77.9 / -; with 8 children (R-MAT scale 18
+// fp32) 4096 took 2.03 ms under the profiler where 8192 takes 1.89, with 16 (scale 19) 21.8 against 21.4 ms per step.
+constexpr int kDirectTileSmall = 4096;
+constexpr int kDirectTileFanout = 32;  // from this fan-out on
+inline int direct_tile(int F) { return F >= kDirectTileFanout ? kDirectTileSmall : kExpandTile; }
+template <typename V, int kDirectTile>
 __global__ void __launch_bounds__(kExpandThreads) k4_expand_direct(
     const i64* __restrict__ seg_off, const i64* __restrict__ seg_bstart, const i64* __restrict__ seg_j,
     const TileMeta* __restrict__ tile_meta,  // per tile: first segment and number of segments
