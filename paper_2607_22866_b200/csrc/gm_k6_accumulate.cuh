@@ -15,16 +15,17 @@
 // that has to synchronise for it.  So the chunks are binned by size (the binning of Section III-E) and
 // every bin gets a team of its own width:
 //   k6_classify      one thread per chunk: lists of the mid-size and of the big chunks
-//   k6_small_chunks  n <= 512 products: one warp per chunk, register sort, no barrier at all
+//   k6_small_chunks  n <= 128 products (an option, at most 512): one warp per chunk, register sort, no barrier at all
 //   k6_mid_chunks    n <= a few thousand: one 128-thread block per chunk, several blocks per SM.  Symbolic
 //                    then numeric as in Algorithm 3: pass 1 sets the column bitmap, a prefix sum over the
 //                    bitmap words ranks the columns, pass 2 adds every product to a *compact* array of the
-//                    chunk's entries (its size is bounded by the chunk's products, not by W, which is what
-//                    lets many chunks share an SM); the second pass re-reads the chunk from L2
+//                    chunk's entries and notes its column in a second one (their size is bounded by the chunk's
+//                    products, not by W, which is what lets many chunks share an SM), the write-out is a plain
+//                    copy of the two; the second pass re-reads the chunk from L2
 //   k6_accumulate    the rest: one 1024-thread block per SM with the dense W-column accumulator, products
 //                    streamed from HBM with 16-byte loads one tile ahead in registers, one flush per chunk
-// All of them are persistent grids that take chunks from a list with an atomic ticket; nothing waits on
-// anything but block-wide barriers.
+// The mid-size and the big kernel are persistent grids that take chunks from a list with an atomic ticket, the
+// small one shares the chunk table out statically; nothing waits on anything but block-wide barriers.
 #pragma once
 #include "gm_common.cuh"
 
@@ -121,7 +122,7 @@ __global__ void k6_chunk_bases(const i64* __restrict__ chunk_nnz_off, i64 n_chun
 
 // Small chunks.  Going through the block-wide accumulator costs every chunk a few thousand cycles of barriers,
 // prefix sums and dependent shared-memory round trips whatever it holds, and most chunks of a power-law product
-// hold few products.  Chunks of at most kAccSmallChunk products are therefore handled before the streaming
+// hold few products.  Chunks of at most small_max (<= kAccSmallChunk) products are therefore handled before the streaming
 // kernel runs, by ONE warp each and with no block-wide step, so that every SM works on dozens of them at a
 // time: the warp loads the chunk, sorts (column, position) keys packed into one word in registers (bitonic
 // network of ascending-only comparators: one shuffle and one min/max per key and step), adds up runs of equal
